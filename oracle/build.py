@@ -1,0 +1,29 @@
+"""Builds the oracle (test infrastructure) into a shared library with the host compiler.
+
+Flags: -O2 (as it stands, never tuned), -ffp-contract=off so that no multiply-add is fused and every
+fp32 operation rounds once, as the block rules require.
+"""
+import os
+import subprocess
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(HERE, "ccz_oracle.cpp")
+HDR = os.path.join(HERE, "ccz_oracle.h")
+LIB = os.path.join(HERE, "libccz_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle/ccz_oracle.cpp if the library is missing or older than its sources."""
+    if not force and os.path.exists(LIB):
+        t = os.path.getmtime(LIB)
+        if t >= os.path.getmtime(SRC) and t >= os.path.getmtime(HDR):
+            return LIB
+    cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-Wall", "-Wextra",
+           "-shared", "-fPIC", SRC, "-o", LIB + ".tmp"]
+    subprocess.run(cmd, check=True, cwd=HERE)
+    os.replace(LIB + ".tmp", LIB)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build(force=True))

@@ -1,0 +1,129 @@
+"""ctypes access to the oracle library (oracle/ccz_oracle.cpp).  TEST INFRASTRUCTURE ONLY.
+
+Numpy arrays in, numpy arrays out; argument marshalling only, no arithmetic of the method lives here.
+"""
+import ctypes
+import numpy as np
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_CORRUPT = 0, 1, 3, 4
+BLOCK_CONSTANT, BLOCK_TRUNCATED, BLOCK_LOSSLESS = 0, 1, 2
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(_build.build())
+        sz, u32, u64, f32, i32, vp = (ctypes.c_size_t, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float,
+                                      ctypes.c_int, ctypes.c_void_p)
+        L.ccz_compress_bound.restype = sz
+        L.ccz_compress_bound.argtypes = [sz, u32]
+        L.ccz_chunk_len.restype = sz
+        L.ccz_chunk_len.argtypes = [sz, i32, u32]
+        L.ccz_quantise_only.restype = i32
+        L.ccz_quantise_only.argtypes = [vp, sz, f32, u32, vp, vp]
+        L.ccz_compress.restype = i32
+        L.ccz_compress.argtypes = [vp, sz, f32, u32, vp, sz, vp]
+        for name in ("ccz_decompress", "ccz_decompress_sequential"):
+            fn = getattr(L, name)
+            fn.restype = i32
+            fn.argtypes = [vp, sz, sz, u32, vp]
+        L.ccz_reduce_step.restype = i32
+        L.ccz_reduce_step.argtypes = [vp, sz, vp, sz, f32, u32, vp, sz, vp, vp]
+        L.ccz_allreduce_sim.restype = i32
+        L.ccz_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp]
+        L.ccz_bcast_sim.restype = i32
+        L.ccz_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp]
+        _lib = L
+    return _lib
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code):
+        super().__init__(f"oracle returned status {code}")
+        self.code = code
+
+
+def _check(rc):
+    if rc != OK:
+        raise OracleError(rc)
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def compress_bound(n, block_len=128):
+    return int(lib().ccz_compress_bound(n, block_len))
+
+
+def chunk_len(n, P, block_len=128):
+    return int(lib().ccz_chunk_len(n, P, block_len))
+
+
+def quantise_only(x, eb, block_len=128):
+    x = _f32(x)
+    xhat = np.empty_like(x)
+    types = np.zeros((x.size + block_len - 1) // block_len, dtype=np.uint8)
+    _check(lib().ccz_quantise_only(_ptr(x), x.size, eb, block_len, _ptr(xhat), _ptr(types)))
+    return xhat, types
+
+
+def compress(x, eb, block_len=128, cap=None):
+    x = _f32(x)
+    if cap is None:
+        cap = compress_bound(x.size, block_len)
+    out = np.zeros(cap, dtype=np.uint8)
+    nbytes = ctypes.c_uint64(0)
+    _check(lib().ccz_compress(_ptr(x), x.size, eb, block_len, _ptr(out), cap, ctypes.byref(nbytes)))
+    return out[: nbytes.value].copy()
+
+
+def decompress(stream, n, block_len=128, sequential=False):
+    stream = np.ascontiguousarray(stream, dtype=np.uint8)
+    out = np.empty(n, dtype=np.float32)
+    fn = lib().ccz_decompress_sequential if sequential else lib().ccz_decompress
+    _check(fn(_ptr(stream), stream.size, n, block_len, _ptr(out)))
+    return out
+
+
+def reduce_step(stream, local, eb, block_len=128, want_sum=False):
+    stream = np.ascontiguousarray(stream, dtype=np.uint8)
+    local = _f32(local)
+    cap = compress_bound(local.size, block_len)
+    out = np.zeros(cap, dtype=np.uint8)
+    nbytes = ctypes.c_uint64(0)
+    s = np.empty_like(local) if want_sum else None
+    _check(lib().ccz_reduce_step(_ptr(stream), stream.size, _ptr(local), local.size, eb, block_len, _ptr(out), cap,
+                                 ctypes.byref(nbytes), _ptr(s) if want_sum else None))
+    return (out[: nbytes.value].copy(), s) if want_sum else out[: nbytes.value].copy()
+
+
+def allreduce_sim(x, eb, block_len=128):
+    """x: [P, n] fp32.  Returns (out [P, n], bytes_moved)."""
+    x = _f32(x)
+    P, n = x.shape
+    out = np.empty_like(x)
+    moved = ctypes.c_uint64(0)
+    _check(lib().ccz_allreduce_sim(_ptr(x), _ptr(out), P, n, eb, block_len, ctypes.byref(moved)))
+    return out, moved.value
+
+
+def bcast_sim(root, P, eb, block_len=128, mode=0):
+    """root: [n] fp32.  mode 0 = BCAST -> out [P, n]; mode 1 = SCATTER -> out [P, chunk_len] (tail unused = 0).
+    Returns (out, chunk_bytes [P])."""
+    root = _f32(root)
+    n = root.size
+    stride = n if mode == 0 else chunk_len(n, P, block_len)
+    out = np.zeros((P, stride), dtype=np.float32)
+    cb = np.zeros(P, dtype=np.uint64)
+    _check(lib().ccz_bcast_sim(_ptr(root), _ptr(out), stride, P, n, eb, block_len, mode, _ptr(cb)))
+    return out, cb

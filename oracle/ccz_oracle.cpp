@@ -1,0 +1,540 @@
+/*
+ * ccz_oracle.cpp — see ccz_oracle.h.  TEST INFRASTRUCTURE ONLY: single thread, no blocking, no fusion,
+ * no intrinsics.  Every routine is written in the order the rules are stated so that it can be checked
+ * against them by eye.
+ *
+ * Block rules (one block = m <= L consecutive values x_0 .. x_{m-1}); the paper (Sec. III-C) only names
+ * the compressor family, so these rules are this project's definition:
+ *   R1  any value with an all-ones exponent (NaN / Inf)            -> LOSSLESS block
+ *   R2  mn, mx = min, max;  mu = 0.5f*mn + 0.5f*mx;  mu == 0 -> mu = +0.0f
+ *   R3  r = max( fl(mx - mu), fl(mu - mn) )
+ *   R4  r <= eb                                                    -> CONSTANT block, payload = mu
+ *   R5  m_bits = E(r) - E(eb) + 1  (E = biased exponent field);  m_bits >= 23 -> LOSSLESS
+ *       else R = 9 + m_bits, B = ceil(R/8), v_i = fl(x_i - mu), q_i = bits(v_i) >> (32 - R)
+ *   R6  LOSSLESS: R = 32, B = 4, stored mu = +0.0f, q_i = bits(x_i)
+ *   R7  lead_i = min(3, B, number of equal most-significant bytes (of the B-byte field) of q_i and
+ *       q_{i-1}), q_{-1} = 0;  element i stores bytes lead_i .. B-1 of q_i, most significant first
+ *   R8  record = [mu f32][R u8][2-bit lead codes, 4 per byte, element i at bits 2(i%4)][stored bytes]
+ *   R9  decode: x^_i = bits-as-float(q_i) if R == 32 else fl( bits-as-float(q_i << (32-R)) + mu )
+ *
+ * Stream layout "CCZ1" (little endian), nb = ceil(n/L) blocks, G = ceil(nb/32) groups of 32 blocks:
+ *   0  u32 magic 0x315A4343   4 u32 flags=0   8 u64 n   16 u32 L   20 f32 eb   24 u64 total_bytes
+ *   32 u32 dir[G+1]  (start of group g's payload in 4-byte words from payload_base; dir[G] = total)
+ *      u32 bitmap[G] (bit i of word g set iff block 32g+i is not CONSTANT)
+ *      zero pad to a multiple of 16 -> payload_base
+ *   group payload: u16 size of every non-constant record, in block order; the records of the group's
+ *      blocks in block order (CONSTANT: 4 bytes mu); zero pad to a multiple of 4.
+ * The index in front of the data follows Sec. III-E-2 (sizes table at the front of the buffer).
+ */
+#include "ccz_oracle.h"
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+constexpr uint32_t kMagic = 0x315A4343u; /* "CCZ1" */
+constexpr size_t kHeaderBytes = 32;
+constexpr uint32_t kBlocksPerGroup = 32;
+
+inline uint32_t bits_of(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  return u;
+}
+inline float float_of(uint32_t u) {
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+inline uint32_t exponent_field(float f) { return (bits_of(f) >> 23) & 0xFFu; }
+
+inline void put_u16(uint8_t* p, uint32_t v) {
+  p[0] = (uint8_t)(v & 0xFF);
+  p[1] = (uint8_t)((v >> 8) & 0xFF);
+}
+inline void put_u32(uint8_t* p, uint32_t v) {
+  for (int k = 0; k < 4; ++k) p[k] = (uint8_t)((v >> (8 * k)) & 0xFF);
+}
+inline void put_u64(uint8_t* p, uint64_t v) {
+  for (int k = 0; k < 8; ++k) p[k] = (uint8_t)((v >> (8 * k)) & 0xFF);
+}
+inline uint32_t get_u16(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8); }
+inline uint32_t get_u32(const uint8_t* p) {
+  uint32_t v = 0;
+  for (int k = 0; k < 4; ++k) v |= (uint32_t)p[k] << (8 * k);
+  return v;
+}
+inline uint64_t get_u64(const uint8_t* p) {
+  uint64_t v = 0;
+  for (int k = 0; k < 8; ++k) v |= (uint64_t)p[k] << (8 * k);
+  return v;
+}
+
+bool valid_block_len(uint32_t L) { return L >= 4 && L <= 1024 && (L % 4) == 0; }
+bool valid_eb(float eb) { return std::isfinite(eb) && eb > 0.0f && exponent_field(eb) >= 1; }
+
+size_t num_blocks(size_t n, uint32_t L) { return (n + L - 1) / L; }
+size_t num_groups(size_t n, uint32_t L) { return (num_blocks(n, L) + kBlocksPerGroup - 1) / kBlocksPerGroup; }
+size_t payload_base(size_t G) {
+  size_t front = kHeaderBytes + 4 * (G + 1) + 4 * G;
+  return (front + 15) / 16 * 16;
+}
+
+/* Rules R1-R6 for one block: decides the type and the parameters (mu, R). */
+struct BlockPlan {
+  int type;   /* CCZ_BLOCK_* */
+  float mu;   /* representative value (0 for LOSSLESS) */
+  uint32_t R; /* kept bits per value (32 for LOSSLESS, unused for CONSTANT) */
+};
+
+BlockPlan plan_block(const float* x, size_t m, float eb) {
+  BlockPlan p;
+  /* R1 */
+  for (size_t i = 0; i < m; ++i) {
+    if (exponent_field(x[i]) == 255u) {
+      p.type = CCZ_BLOCK_LOSSLESS;
+      p.mu = 0.0f;
+      p.R = 32;
+      return p;
+    }
+  }
+  /* R2 */
+  float mn = x[0], mx = x[0];
+  for (size_t i = 1; i < m; ++i) {
+    if (x[i] < mn) mn = x[i];
+    if (x[i] > mx) mx = x[i];
+  }
+  float half_mn = 0.5f * mn;
+  float half_mx = 0.5f * mx;
+  float mu = half_mn + half_mx;
+  if (mu == 0.0f) mu = float_of(0u); /* a zero of either sign becomes +0 */
+  /* R3 */
+  float up = mx - mu;
+  float dn = mu - mn;
+  float r = (up > dn) ? up : dn;
+  /* R4 */
+  if (r <= eb) {
+    p.type = CCZ_BLOCK_CONSTANT;
+    p.mu = mu;
+    p.R = 0;
+    return p;
+  }
+  /* R5 */
+  int m_bits = (int)exponent_field(r) - (int)exponent_field(eb) + 1;
+  if (m_bits >= 23) {
+    p.type = CCZ_BLOCK_LOSSLESS;
+    p.mu = 0.0f;
+    p.R = 32;
+    return p;
+  }
+  p.type = CCZ_BLOCK_TRUNCATED;
+  p.mu = mu;
+  p.R = (uint32_t)(9 + m_bits);
+  return p;
+}
+
+/* R5/R6: the integer code of one value. */
+inline uint32_t code_of(float x, const BlockPlan& p) {
+  if (p.R == 32) return bits_of(x);
+  float v = x - p.mu;
+  return bits_of(v) >> (32 - p.R);
+}
+/* R9: the value a code stands for. */
+inline float value_of(uint32_t q, float mu, uint32_t R) {
+  if (R == 32) return float_of(q);
+  float v = float_of(q << (32 - R));
+  return v + mu;
+}
+
+/* R7: number of leading (most significant) bytes, out of B, that cur shares with prev; capped at 3. */
+inline uint32_t lead_bytes(uint32_t cur, uint32_t prev, uint32_t B) {
+  uint32_t lead = 0;
+  while (lead < B && lead < 3) {
+    uint32_t shift = 8 * (B - 1 - lead);
+    if (((cur >> shift) & 0xFFu) != ((prev >> shift) & 0xFFu)) break;
+    ++lead;
+  }
+  return lead;
+}
+
+/* R7/R8: append the record of a non-constant block to `rec`. */
+void encode_record(const float* x, size_t m, const BlockPlan& p, std::vector<uint8_t>& rec) {
+  uint32_t B = (p.R + 7) / 8;
+  size_t code_bytes = (m + 3) / 4;
+  size_t start = rec.size();
+  rec.resize(start + 5 + code_bytes, 0);
+  put_u32(&rec[start], bits_of(p.mu));
+  rec[start + 4] = (uint8_t)p.R;
+  uint32_t prev = 0;
+  for (size_t i = 0; i < m; ++i) {
+    uint32_t q = code_of(x[i], p);
+    uint32_t lead = lead_bytes(q, prev, B);
+    rec[start + 5 + i / 4] |= (uint8_t)(lead << (2 * (i % 4)));
+    for (uint32_t j = lead; j < B; ++j) rec.push_back((uint8_t)((q >> (8 * (B - 1 - j))) & 0xFFu));
+    prev = q;
+  }
+}
+
+/* R9 with full validation: decode one non-constant record of exactly `size` bytes holding m values. */
+int decode_record(const uint8_t* rec, size_t size, size_t m, float* out) {
+  size_t code_bytes = (m + 3) / 4;
+  if (size < 5 + code_bytes) return CCZ_ERR_CORRUPT;
+  float mu = float_of(get_u32(rec));
+  uint32_t R = rec[4];
+  if (!((R >= 10 && R <= 31) || R == 32)) return CCZ_ERR_CORRUPT;
+  uint32_t B = (R + 7) / 8;
+  const uint8_t* codes = rec + 5;
+  size_t pos = 5 + code_bytes;
+  uint32_t prev = 0;
+  for (size_t i = 0; i < m; ++i) {
+    uint32_t lead = (codes[i / 4] >> (2 * (i % 4))) & 3u;
+    if (lead > B) return CCZ_ERR_CORRUPT;
+    uint32_t q = 0;
+    for (uint32_t j = 0; j < B; ++j) {
+      uint32_t shift = 8 * (B - 1 - j);
+      uint32_t byte;
+      if (j < lead) {
+        byte = (prev >> shift) & 0xFFu;
+      } else {
+        if (pos >= size) return CCZ_ERR_CORRUPT;
+        byte = rec[pos++];
+      }
+      q |= byte << shift;
+    }
+    out[i] = value_of(q, mu, R);
+    prev = q;
+  }
+  /* unused code bits must be zero and the record must be used up exactly */
+  for (size_t i = m; i < 4 * code_bytes; ++i)
+    if ((codes[i / 4] >> (2 * (i % 4))) & 3u) return CCZ_ERR_CORRUPT;
+  if (pos != size) return CCZ_ERR_CORRUPT;
+  return CCZ_OK;
+}
+
+struct Header {
+  uint64_t n;
+  uint32_t L;
+  float eb;
+  uint64_t total;
+  size_t G;
+  size_t base;
+};
+
+int parse_header(const uint8_t* in, size_t in_bytes, size_t n, uint32_t L, Header& h) {
+  if (!in || !valid_block_len(L)) return CCZ_ERR_INVALID_ARG;
+  if (in_bytes < kHeaderBytes) return CCZ_ERR_CORRUPT;
+  if (get_u32(in) != kMagic || get_u32(in + 4) != 0u) return CCZ_ERR_CORRUPT;
+  h.n = get_u64(in + 8);
+  h.L = get_u32(in + 16);
+  h.eb = float_of(get_u32(in + 20));
+  h.total = get_u64(in + 24);
+  if (h.n != (uint64_t)n || h.L != L) return CCZ_ERR_CORRUPT;
+  h.G = num_groups(n, L);
+  h.base = payload_base(h.G);
+  if (h.total > in_bytes || h.total < h.base) return CCZ_ERR_CORRUPT;
+  return CCZ_OK;
+}
+
+/* Decode group g whose payload is [p, p+bytes). */
+int decode_group(const uint8_t* p, size_t bytes, uint32_t bitmap, size_t g, size_t n, uint32_t L, float* out) {
+  size_t nb = num_blocks(n, L);
+  size_t first = g * kBlocksPerGroup;
+  size_t count = (nb - first < kBlocksPerGroup) ? nb - first : kBlocksPerGroup;
+  if (count < 32 && (bitmap >> count) != 0u) return CCZ_ERR_CORRUPT;
+  uint32_t k = 0;
+  for (size_t b = 0; b < count; ++b) k += (bitmap >> b) & 1u;
+  if (bytes < 2 * (size_t)k) return CCZ_ERR_CORRUPT;
+  size_t pos = 2 * (size_t)k;
+  uint32_t j = 0;
+  for (size_t b = 0; b < count; ++b) {
+    size_t blk = first + b;
+    size_t m = (blk + 1) * (size_t)L <= n ? L : n - blk * (size_t)L;
+    float* dst = out + blk * (size_t)L;
+    if ((bitmap >> b) & 1u) {
+      size_t size = get_u16(p + 2 * j);
+      ++j;
+      if (pos + size > bytes) return CCZ_ERR_CORRUPT;
+      int rc = decode_record(p + pos, size, m, dst);
+      if (rc != CCZ_OK) return rc;
+      pos += size;
+    } else {
+      if (pos + 4 > bytes) return CCZ_ERR_CORRUPT;
+      float mu = float_of(get_u32(p + pos));
+      for (size_t i = 0; i < m; ++i) dst[i] = mu;
+      pos += 4;
+    }
+  }
+  size_t padded = (pos + 3) / 4 * 4;
+  if (padded != bytes) return CCZ_ERR_CORRUPT;
+  for (size_t q = pos; q < padded; ++q)
+    if (p[q] != 0) return CCZ_ERR_CORRUPT;
+  return CCZ_OK;
+}
+
+} /* namespace */
+
+extern "C" {
+
+size_t ccz_compress_bound(size_t n, uint32_t L) {
+  if (!valid_block_len(L)) return 0;
+  size_t G = num_groups(n, L);
+  size_t max_record = 5 + L / 4 + 4 * (size_t)L;
+  size_t max_group = 2 * kBlocksPerGroup + kBlocksPerGroup * max_record + 3;
+  return kHeaderBytes + 4 * (G + 1) + 4 * G + 15 + G * max_group;
+}
+
+size_t ccz_chunk_len(size_t n, int P, uint32_t L) {
+  if (P < 1 || !valid_block_len(L)) return 0;
+  size_t per = (n + (size_t)P - 1) / (size_t)P;
+  return (per + L - 1) / L * L;
+}
+
+int ccz_quantise_only(const float* x, size_t n, float eb, uint32_t L, float* xhat, uint8_t* block_type) {
+  if ((!x || !xhat) && n) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  size_t nb = num_blocks(n, L);
+  for (size_t b = 0; b < nb; ++b) {
+    size_t off = b * (size_t)L;
+    size_t m = (off + L <= n) ? L : n - off;
+    BlockPlan p = plan_block(x + off, m, eb);
+    if (block_type) block_type[b] = (uint8_t)p.type;
+    for (size_t i = 0; i < m; ++i) {
+      if (p.type == CCZ_BLOCK_CONSTANT) {
+        xhat[off + i] = p.mu;
+      } else {
+        xhat[off + i] = value_of(code_of(x[off + i], p), p.mu, p.R);
+      }
+    }
+  }
+  return CCZ_OK;
+}
+
+int ccz_compress(const float* x, size_t n, float eb, uint32_t L, uint8_t* out, size_t cap, uint64_t* out_bytes) {
+  if (!out || !out_bytes || (!x && n)) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  size_t nb = num_blocks(n, L);
+  size_t G = num_groups(n, L);
+  size_t base = payload_base(G);
+  if (cap < base) return CCZ_ERR_CAPACITY;
+  std::memset(out, 0, base);
+  uint8_t* dir = out + kHeaderBytes;
+  uint8_t* bitmap = dir + 4 * (G + 1);
+  size_t pos = base; /* byte position of the next group payload */
+  std::vector<uint8_t> sizes, records;
+  for (size_t g = 0; g < G; ++g) {
+    put_u32(dir + 4 * g, (uint32_t)((pos - base) / 4));
+    size_t first = g * kBlocksPerGroup;
+    size_t count = (nb - first < kBlocksPerGroup) ? nb - first : kBlocksPerGroup;
+    uint32_t map = 0;
+    sizes.clear();
+    records.clear();
+    for (size_t b = 0; b < count; ++b) {
+      size_t off = (first + b) * (size_t)L;
+      size_t m = (off + L <= n) ? L : n - off;
+      BlockPlan p = plan_block(x + off, m, eb);
+      if (p.type == CCZ_BLOCK_CONSTANT) {
+        size_t s = records.size();
+        records.resize(s + 4);
+        put_u32(&records[s], bits_of(p.mu));
+      } else {
+        map |= 1u << b;
+        size_t before = records.size();
+        encode_record(x + off, m, p, records);
+        size_t rec_size = records.size() - before;
+        size_t s = sizes.size();
+        sizes.resize(s + 2);
+        put_u16(&sizes[s], (uint32_t)rec_size);
+      }
+    }
+    put_u32(bitmap + 4 * g, map);
+    size_t raw = sizes.size() + records.size();
+    size_t padded = (raw + 3) / 4 * 4;
+    if (pos + padded > cap) return CCZ_ERR_CAPACITY;
+    if (!sizes.empty()) std::memcpy(out + pos, sizes.data(), sizes.size());
+    if (!records.empty()) std::memcpy(out + pos + sizes.size(), records.data(), records.size());
+    for (size_t q = raw; q < padded; ++q) out[pos + q] = 0;
+    pos += padded;
+  }
+  put_u32(dir + 4 * G, (uint32_t)((pos - base) / 4));
+  put_u32(out + 0, kMagic);
+  put_u32(out + 4, 0u);
+  put_u64(out + 8, (uint64_t)n);
+  put_u32(out + 16, L);
+  put_u32(out + 20, bits_of(eb));
+  put_u64(out + 24, (uint64_t)pos);
+  *out_bytes = (uint64_t)pos;
+  return CCZ_OK;
+}
+
+int ccz_decompress(const uint8_t* in, size_t in_bytes, size_t n, uint32_t L, float* out) {
+  Header h;
+  int rc = parse_header(in, in_bytes, n, L, h);
+  if (rc != CCZ_OK) return rc;
+  if (!out && n) return CCZ_ERR_INVALID_ARG;
+  const uint8_t* dir = in + kHeaderBytes;
+  const uint8_t* bitmap = dir + 4 * (h.G + 1);
+  size_t payload_bytes = h.total - h.base;
+  if (payload_bytes % 4) return CCZ_ERR_CORRUPT;
+  if ((uint64_t)get_u32(dir + 4 * h.G) * 4 != payload_bytes) return CCZ_ERR_CORRUPT;
+  for (size_t q = kHeaderBytes + 8 * h.G + 4; q < h.base; ++q)
+    if (in[q] != 0) return CCZ_ERR_CORRUPT;
+  for (size_t g = 0; g < h.G; ++g) {
+    uint64_t a = (uint64_t)get_u32(dir + 4 * g) * 4;
+    uint64_t b = (uint64_t)get_u32(dir + 4 * (g + 1)) * 4;
+    if (a > b || b > payload_bytes) return CCZ_ERR_CORRUPT;
+    rc = decode_group(in + h.base + a, (size_t)(b - a), get_u32(bitmap + 4 * g), g, n, L, out);
+    if (rc != CCZ_OK) return rc;
+  }
+  return CCZ_OK;
+}
+
+int ccz_decompress_sequential(const uint8_t* in, size_t in_bytes, size_t n, uint32_t L, float* out) {
+  Header h;
+  int rc = parse_header(in, in_bytes, n, L, h);
+  if (rc != CCZ_OK) return rc;
+  if (!out && n) return CCZ_ERR_INVALID_ARG;
+  const uint8_t* dir = in + kHeaderBytes;
+  const uint8_t* bitmap = dir + 4 * (h.G + 1);
+  size_t nb = num_blocks(n, L);
+  size_t pos = h.base; /* walks the payload byte by byte; never reads dir[] to find a group */
+  size_t j = 0;        /* index into the current group's size table */
+  size_t table = 0;    /* position of the current group's size table */
+  for (size_t blk = 0; blk < nb; ++blk) {
+    size_t g = blk / kBlocksPerGroup, b = blk % kBlocksPerGroup;
+    uint32_t map = get_u32(bitmap + 4 * g);
+    if (b == 0) {
+      /* a new group begins: realign, check the directory agrees, skip over its size table */
+      pos = (pos + 3) / 4 * 4;
+      if ((uint64_t)get_u32(dir + 4 * g) * 4 != pos - h.base) return CCZ_ERR_CORRUPT;
+      uint32_t k = 0;
+      for (uint32_t t = 0; t < kBlocksPerGroup; ++t) k += (map >> t) & 1u;
+      table = pos;
+      j = 0;
+      pos += 2 * (size_t)k;
+      if (pos > h.total) return CCZ_ERR_CORRUPT;
+    }
+    size_t m = (blk + 1) * (size_t)L <= n ? L : n - blk * (size_t)L;
+    float* dst = out + blk * (size_t)L;
+    if ((map >> b) & 1u) {
+      size_t size = get_u16(in + table + 2 * j);
+      ++j;
+      if (pos + size > h.total) return CCZ_ERR_CORRUPT;
+      rc = decode_record(in + pos, size, m, dst);
+      if (rc != CCZ_OK) return rc;
+      pos += size;
+    } else {
+      if (pos + 4 > h.total) return CCZ_ERR_CORRUPT;
+      float mu = float_of(get_u32(in + pos));
+      for (size_t i = 0; i < m; ++i) dst[i] = mu;
+      pos += 4;
+    }
+  }
+  pos = (pos + 3) / 4 * 4;
+  if (pos != h.total) return CCZ_ERR_CORRUPT;
+  if ((uint64_t)get_u32(dir + 4 * h.G) * 4 != pos - h.base) return CCZ_ERR_CORRUPT;
+  return CCZ_OK;
+}
+
+int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L,
+                    uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
+  if (!local && n) return CCZ_ERR_INVALID_ARG;
+  std::vector<float> s(n);
+  int rc = ccz_decompress(in, in_bytes, n, L, s.data());
+  if (rc != CCZ_OK) return rc;
+  for (size_t i = 0; i < n; ++i) s[i] = s[i] + local[i];
+  rc = ccz_compress(s.data(), n, eb, L, out, cap, out_bytes);
+  if (rc != CCZ_OK) return rc;
+  if (sum_out)
+    for (size_t i = 0; i < n; ++i) sum_out[i] = s[i];
+  return CCZ_OK;
+}
+
+int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, uint32_t L, uint64_t* bytes_moved) {
+  if (P < 1 || ((!in || !out) && n)) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  size_t C = ccz_chunk_len(n, P, L);
+  uint64_t moved = 0;
+  std::vector<uint8_t> sa, sb;
+  std::vector<float> dec;
+  for (int c = 0; c < P; ++c) {
+    size_t lo = (size_t)c * C < n ? (size_t)c * C : n;
+    size_t hi = (size_t)(c + 1) * C < n ? (size_t)(c + 1) * C : n;
+    size_t len = hi - lo;
+    if (P == 1) { /* a single rank keeps its own data; nothing is sent */
+      for (size_t i = 0; i < len; ++i) out[lo + i] = in[lo + i];
+      continue;
+    }
+    size_t cap = ccz_compress_bound(len, L);
+    sa.assign(cap, 0);
+    sb.assign(cap, 0);
+    dec.assign(len, 0.0f);
+    /* round 0: rank c compresses its own chunk c and sends it to rank c+1 */
+    uint64_t bytes = 0;
+    int rc = ccz_compress(in + (size_t)c * n + lo, len, eb, L, sa.data(), cap, &bytes);
+    if (rc != CCZ_OK) return rc;
+    moved += bytes;
+    /* rounds 1..P-1 (Fig. 4): rank (c+k) mod P decompresses, adds its chunk c, recompresses */
+    int owner = (c + P - 1) % P;
+    for (int k = 1; k <= P - 1; ++k) {
+      int r = (c + k) % P;
+      uint64_t nbytes = 0;
+      float* sum_out = (k == P - 1) ? out + (size_t)owner * n + lo : nullptr;
+      rc = ccz_reduce_step(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, sb.data(), cap, &nbytes,
+                           sum_out);
+      if (rc != CCZ_OK) return rc;
+      sa.swap(sb);
+      bytes = nbytes;
+      if (k < P - 1) moved += bytes;
+    }
+    /* allgather (Sec. III-E-1): the final stream travels P-1 hops; every rank except its owner decodes it */
+    moved += (uint64_t)(P - 1) * bytes;
+    rc = ccz_decompress(sa.data(), (size_t)bytes, len, L, dec.data());
+    if (rc != CCZ_OK) return rc;
+    for (int r = 0; r < P; ++r) {
+      if (r == owner) continue;
+      for (size_t i = 0; i < len; ++i) out[(size_t)r * n + lo + i] = dec[i];
+    }
+  }
+  if (bytes_moved) *bytes_moved = moved;
+  return CCZ_OK;
+}
+
+int ccz_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float eb, uint32_t L,
+                  int mode, uint64_t* chunk_bytes) {
+  if (P < 1 || ((!root_in || !out) && n) || (mode != 0 && mode != 1)) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  size_t C = ccz_chunk_len(n, P, L);
+  std::vector<uint8_t> stream;
+  std::vector<float> dec;
+  for (int c = 0; c < P; ++c) {
+    size_t lo = (size_t)c * C < n ? (size_t)c * C : n;
+    size_t hi = (size_t)(c + 1) * C < n ? (size_t)(c + 1) * C : n;
+    size_t len = hi - lo;
+    /* the root compresses every chunk exactly once (Sec. III-A-1) */
+    size_t cap = ccz_compress_bound(len, L);
+    stream.assign(cap, 0);
+    uint64_t bytes = 0;
+    int rc = ccz_compress(root_in + lo, len, eb, L, stream.data(), cap, &bytes);
+    if (rc != CCZ_OK) return rc;
+    if (chunk_bytes) chunk_bytes[c] = bytes;
+    dec.assign(len, 0.0f);
+    rc = ccz_decompress(stream.data(), (size_t)bytes, len, L, dec.data());
+    if (rc != CCZ_OK) return rc;
+    if (mode == 1) {
+      /* SCATTER: rank c receives chunk c; the root keeps its own chunk as it is */
+      float* dst = out + (size_t)c * out_rank_stride;
+      for (size_t i = 0; i < len; ++i) dst[i] = (c == 0) ? root_in[lo + i] : dec[i];
+    } else {
+      /* BCAST: every rank receives every chunk; the root keeps its original buffer */
+      for (int r = 0; r < P; ++r) {
+        float* dst = out + (size_t)r * out_rank_stride + lo;
+        for (size_t i = 0; i < len; ++i) dst[i] = (r == 0) ? root_in[lo + i] : dec[i];
+      }
+    }
+  }
+  return CCZ_OK;
+}
+
+} /* extern "C" */

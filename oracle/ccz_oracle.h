@@ -1,0 +1,95 @@
+/*
+ * ccz_oracle.h — reference ("oracle") implementation of the C-Coll hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, single-threaded, deliberately slow C++17 program that
+ * states what the CUDA library must compute.  It shares no code with the CUDA path and is never called
+ * by it; only the test-suite, the smoke check and the CPU-baseline leg of the benchmark may use it.
+ *
+ * What it follows in the paper (arXiv 2304.03890, "C-Coll"):
+ *   - Sec. III-C / Table I: the compressor is an error-bounded (absolute bound), 1-D, fp32 compressor of
+ *     the SZx family.  The paper cites that compressor but does not define its internals, so the block
+ *     rules and the byte layout below are this project's own definition ("CCZ1").
+ *   - Sec. III-E-2 (PIPE-SZx): compressed pieces have variable length, so an index is kept at the FRONT of
+ *     the output buffer instead of between the pieces.  Here the pieces are groups of 32 blocks and the
+ *     index stores offsets (the running sum of the sizes) so a decoder needs no scan.
+ *   - Sec. III-A-1 / III-E-1 (collective data movement framework): a chunk is compressed once by its owner,
+ *     forwarded compressed, decompressed once by every receiver; the owner never decompresses its own.
+ *   - Sec. III-A-2, Fig. 4 (collective computation framework): ring reduce-scatter where every round
+ *     decompresses the received chunk, reduces it with the local chunk and recompresses the result; the
+ *     chunk is the input divided by the number of processes.
+ *   - Sec. III-B: same error bound on every rank and round; data-movement error stays within the bound.
+ *
+ * Parity pins (tests, CPU only): a hand-worked 4-value stream, the error-bound invariant, exact
+ * reproduction of constant blocks, the identity special case (lossless blocks), closed-form stream sizes,
+ * a stream-free closed form of the quantiser (quantise_only), a directory-free sequential decoder
+ * (decompress_sequential), and the P*eb bound of the all-reduce against an fp64 sum.
+ * The compression-ratio envelope of the paper's Table II is only a plausibility report: "parity unpinned"
+ * by it.
+ *
+ * All fp32 arithmetic is IEEE-754 round-to-nearest, no fused multiply-add, no flush-to-zero
+ * (build with -ffp-contract=off).
+ */
+#ifndef CCZ_ORACLE_H
+#define CCZ_ORACLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  CCZ_OK = 0,
+  CCZ_ERR_INVALID_ARG = 1,
+  CCZ_ERR_CAPACITY = 3,
+  CCZ_ERR_CORRUPT = 4
+};
+
+enum { CCZ_BLOCK_CONSTANT = 0, CCZ_BLOCK_TRUNCATED = 1, CCZ_BLOCK_LOSSLESS = 2 };
+
+/* Worst-case stream size for n values in blocks of block_len. */
+size_t ccz_compress_bound(size_t n, uint32_t block_len);
+
+/* Chunk length (in values) used when a buffer of n values is divided among P ranks
+ * (Sec. III-A-2: "dividing the size of the input data by the number of processes"), rounded up to a whole
+ * number of blocks so that every chunk starts on a block boundary. */
+size_t ccz_chunk_len(size_t n, int P, uint32_t block_len);
+
+/* Per-block quantiser without any stream: xhat[i] is the value a decoder must return for x[i];
+ * block_type[b] (nullable) receives CCZ_BLOCK_*. */
+int ccz_quantise_only(const float* x, size_t n, float eb, uint32_t block_len, float* xhat,
+                      uint8_t* block_type);
+
+/* Encode x[0..n) into out (capacity cap bytes); *out_bytes receives the stream length. */
+int ccz_compress(const float* x, size_t n, float eb, uint32_t block_len, uint8_t* out, size_t cap,
+                 uint64_t* out_bytes);
+
+/* Decode using the directory at the front of the stream. */
+int ccz_decompress(const uint8_t* in, size_t in_bytes, size_t n, uint32_t block_len, float* out);
+
+/* Decode by walking the payload front to back, recomputing every offset from the recorded sizes and
+ * using the directory only to cross-check.  Independent of ccz_decompress's offset arithmetic. */
+int ccz_decompress_sequential(const uint8_t* in, size_t in_bytes, size_t n, uint32_t block_len, float* out);
+
+/* One round of the ring reduce-scatter (Fig. 4): decode `in`, add `local` (fp32), encode the sum.
+ * sum_out (nullable) receives the uncompressed sum. */
+int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb,
+                    uint32_t block_len, uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out);
+
+/* C-Allreduce (Sec. III-E) replayed over P virtual ranks: in and out are [P][n], rank-major.
+ * bytes_moved (nullable) = total compressed bytes that would cross the network. */
+int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, uint32_t block_len,
+                      uint64_t* bytes_moved);
+
+/* C-Bcast (mode 0) / C-Scatter (mode 1) over P virtual ranks, root = rank 0.
+ * out_rank_stride is in floats; rank i's output starts at out + i*out_rank_stride.
+ * BCAST: each rank receives n values.  SCATTER: rank i receives its chunk (ccz_chunk_len values or fewer).
+ * chunk_bytes (nullable, [P]) receives the compressed size of every chunk. */
+int ccz_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float eb,
+                  uint32_t block_len, int mode, uint64_t* chunk_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

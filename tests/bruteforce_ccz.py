@@ -1,0 +1,102 @@
+"""A second, deliberately different statement of the CCZ1 block rules for tiny inputs.
+
+Pure Python on hex strings and numpy.float32 scalars: bytes are compared as two-character strings, the
+stream is built as one long hex string.  It exists only so that the oracle's packer can be brute-forced
+against something that shares none of its index arithmetic.  Tiny inputs only (it is very slow).
+"""
+import struct
+
+import numpy as np
+
+f32 = np.float32
+
+
+def hexbits(v) -> str:
+    return struct.pack(">f", float(v)).hex()  # big-endian hex of the fp32 pattern
+
+
+def le(value: int, nbytes: int) -> str:
+    return value.to_bytes(nbytes, "little").hex()
+
+
+def expo(v) -> int:
+    return (int(hexbits(v), 16) >> 23) & 0xFF
+
+
+def block_record(xs, eb):
+    """Returns (is_nonconstant, record hex, decoded values)."""
+    with np.errstate(all="ignore"):
+        special = any(expo(v) == 255 for v in xs)
+        if not special:
+            mn, mx = min(xs), max(xs)
+            mu = f32(f32(0.5) * mn) + f32(f32(0.5) * mx)
+            if mu == 0:
+                mu = f32(0.0)
+            r = max(f32(mx - mu), f32(mu - mn))
+            if r <= eb:
+                return False, bytes.fromhex(hexbits(mu))[::-1].hex(), [mu] * len(xs)
+            mbits = expo(r) - expo(eb) + 1
+        if special or mbits >= 23:
+            R, mu = 32, f32(0.0)
+            fields = [hexbits(v) for v in xs]  # 4 bytes, most significant first
+        else:
+            R = 9 + mbits
+            fields = []
+            for v in xs:
+                q = int(hexbits(f32(v - mu)), 16) >> (32 - R)
+                fields.append(format(q, "0%dx" % (2 * ((R + 7) // 8))))
+    B = (R + 7) // 8
+    codes = [0] * ((len(xs) + 3) // 4)
+    stored = ""
+    prev = "00" * B
+    for i, cur in enumerate(fields):
+        same = 0
+        while same < min(3, B) and cur[2 * same: 2 * same + 2] == prev[2 * same: 2 * same + 2]:
+            same += 1
+        codes[i // 4] += same * 4 ** (i % 4)
+        stored += cur[2 * same:]
+        prev = cur
+    rec = bytes.fromhex(hexbits(mu))[::-1].hex() + le(R, 1) + "".join(le(c, 1) for c in codes) + stored
+    dec = []
+    with np.errstate(all="ignore"):
+        for cur in fields:
+            q = int(cur, 16)
+            if R == 32:
+                dec.append(np.frombuffer(struct.pack("<I", q), dtype=f32)[0])
+            else:
+                dec.append(f32(np.frombuffer(struct.pack("<I", (q << (32 - R)) & 0xFFFFFFFF), dtype=f32)[0] + mu))
+    return True, rec, dec
+
+
+def encode(x, eb, L):
+    """Returns (stream bytes, decoded list) for a small fp32 array."""
+    x = [f32(v) for v in x]
+    eb = f32(eb)
+    n = len(x)
+    blocks = [x[i: i + L] for i in range(0, n, L)]
+    groups = [blocks[i: i + 32] for i in range(0, len(blocks), 32)]
+    G = len(groups)
+    payloads, maps, decoded = [], [], []
+    for grp in groups:
+        table, recs, bits = "", "", 0
+        for b, blk in enumerate(grp):
+            nonconst, rec, dec = block_record(blk, eb)
+            decoded += dec
+            recs += rec
+            if nonconst:
+                bits |= 1 << b
+                table += le(len(rec) // 2, 2)
+        body = table + recs
+        body += "00" * (-(len(body) // 2) % 4)
+        payloads.append(body)
+        maps.append(bits)
+    dirs, words = [], 0
+    for body in payloads:
+        dirs.append(words)
+        words += len(body) // 8
+    dirs.append(words)
+    front = "".join(le(d, 4) for d in dirs) + "".join(le(m, 4) for m in maps)
+    front += "00" * (-(32 + len(front) // 2) % 16)
+    total = 32 + len(front) // 2 + 4 * words
+    header = "43435a31" + le(0, 4) + le(n, 8) + le(L, 4) + bytes.fromhex(hexbits(eb))[::-1].hex() + le(total, 8)
+    return bytes.fromhex(header + front + "".join(payloads)), decoded

@@ -1,0 +1,132 @@
+"""Pins for the oracle's collective replays (CPU only): error laws of Sec. III-B, the compress-once rule of
+Sec. III-A-1, the ring schedule of Sec. III-A-2 / Fig. 4 and the traffic formula of Sec. III-E."""
+import numpy as np
+import pytest
+
+from oracle import ccz
+from paper_2304_03890_b200 import fields
+
+
+def ranks_c3(P, shape=(24, 24, 32)):
+    c = fields.config3(P=P, shape=shape, sigma=3.0)
+    return c["x"].numpy(), np.float32(c["eb"])
+
+
+def test_reduce_step_is_decode_add_encode_within_bound():
+    x, eb = ranks_c3(2)
+    a, b = x[0], x[1]
+    s0 = ccz.compress(a, eb)
+    s1, total = ccz.reduce_step(s0, b, eb, want_sum=True)
+    ahat = ccz.decompress(s0, a.size)
+    # the uncompressed sum is one fp32 add per element
+    assert total.tobytes() == (ahat + b).astype(np.float32).tobytes()
+    d = ccz.decompress(s1, a.size)
+    assert np.abs(d.astype(np.float64) - total.astype(np.float64)).max() <= float(eb)
+    # two lossy passes: within 2 eb of the exact sum
+    exact = a.astype(np.float64) + b.astype(np.float64)
+    assert np.abs(d - exact).max() <= 2 * float(eb) + 2.0 ** -23 * np.abs(exact).max()
+
+
+@pytest.mark.parametrize("P,n", [(2, 5000), (3, 4096 * 3), (4, 128 * 37 + 5), (8, 24 * 24 * 32)])
+def test_allreduce_within_P_eb_of_fp64_sum(P, n):
+    x, eb = ranks_c3(P)
+    x = np.ascontiguousarray(x[:, :n])
+    out, moved = ccz.allreduce_sim(x, eb)
+    exact = x.astype(np.float64).sum(axis=0)
+    slack = P * 2.0 ** -23 * np.abs(exact).max()
+    err = np.abs(out.astype(np.float64) - exact[None, :])
+    assert err.max() <= P * float(eb) + slack
+    # the owner of chunk c is rank c-1: it keeps the uncompressed sum, one lossy pass fewer
+    C = ccz.chunk_len(n, P)
+    for c in range(P):
+        lo, hi = min(n, c * C), min(n, (c + 1) * C)
+        owner = (c - 1) % P
+        assert err[owner, lo:hi].max(initial=0) <= (P - 1) * float(eb) + slack
+        # all the other ranks hold one and the same decoded copy
+        others = [r for r in range(P) if r != owner]
+        for r in others[1:]:
+            assert out[r, lo:hi].tobytes() == out[others[0], lo:hi].tobytes()
+        if hi > lo and P > 1:
+            assert np.abs(out[owner, lo:hi].astype(np.float64) - out[others[0], lo:hi]).max() <= float(eb)
+    # soft check (Corollary 1): most elements within (2/3) sqrt(P) eb — reported, loosely asserted
+    frac = (err <= (2.0 / 3.0) * np.sqrt(P) * float(eb)).mean()
+    assert frac > 0.9
+
+
+def test_allreduce_matches_manual_ring_schedule():
+    """Chunk c starts at rank c and visits ranks c+1, c+2, ... (Fig. 4); replay it with the single-stream
+    routines and compare outputs and the byte count."""
+    P, n = 4, 128 * 50 + 17
+    x, eb = ranks_c3(P)
+    x = np.ascontiguousarray(x[:, :n])
+    out, moved = ccz.allreduce_sim(x, eb)
+    C = ccz.chunk_len(n, P)
+    manual = 0
+    for c in range(P):
+        lo, hi = min(n, c * C), min(n, (c + 1) * C)
+        s = ccz.compress(x[c, lo:hi], eb)
+        manual += s.size
+        for k in range(1, P):
+            r = (c + k) % P
+            s, total = ccz.reduce_step(s, x[r, lo:hi], eb, want_sum=True)
+            if k < P - 1:
+                manual += s.size
+        manual += (P - 1) * s.size
+        owner = (c + P - 1) % P
+        assert out[owner, lo:hi].tobytes() == total.tobytes()
+        dec = ccz.decompress(s, hi - lo)
+        for r in range(P):
+            if r != owner:
+                assert out[r, lo:hi].tobytes() == dec.tobytes()
+    assert moved == manual
+
+
+def test_allreduce_special_cases():
+    # one rank: nothing is sent, the data is untouched
+    x = np.random.default_rng(0).normal(0, 1, (1, 1000)).astype(np.float32)
+    out, moved = ccz.allreduce_sim(x, np.float32(1e-3))
+    assert out.tobytes() == x.tobytes() and moved == 0
+    # identical constant blocks on every rank: the sum is exact
+    P, n = 5, 4096 * 2
+    x = np.full((P, n), 0.75, dtype=np.float32)
+    out, moved = ccz.allreduce_sim(x, np.float32(1e-3))
+    assert np.all(out == np.float32(P * 0.75))
+    # traffic (Sec. III-E): every rank sends 2(P-1)/P * D / CR bytes; with all-constant chunks every stream
+    # has the closed-form size S, so the total over P ranks is 2 P (P-1) S
+    C = ccz.chunk_len(n, P)
+    sizes = []
+    for c in range(P):
+        ln = max(0, min(n, (c + 1) * C) - min(n, c * C))
+        G = (ln + 4095) // 4096
+        nb = (ln + 127) // 128
+        sizes.append((36 + 8 * G + 15) // 16 * 16 + 4 * nb)
+    assert moved == sum(2 * (P - 1) * S for S in sizes)
+
+
+@pytest.mark.parametrize("P", [1, 3, 8])
+def test_bcast_and_scatter(P):
+    c4 = fields.config4(P=P, shape=(16, 32, 40), sigma=3.0)
+    root, eb = c4["x"].numpy()[: 16 * 32 * 40 - 19], np.float32(c4["eb"])
+    n = root.size
+    bc, cb = ccz.bcast_sim(root, P, eb, mode=0)
+    sc, cb2 = ccz.bcast_sim(root, P, eb, mode=1)
+    assert np.array_equal(cb, cb2)
+    # root keeps its buffer; every other rank is within eb (compressed exactly once, Sec. III-B)
+    assert bc[0].tobytes() == root.tobytes()
+    for r in range(1, P):
+        assert np.abs(bc[r].astype(np.float64) - root).max() <= float(eb)
+        assert bc[r].tobytes() == bc[1].tobytes()
+    C = ccz.chunk_len(n, P)
+    for r in range(P):
+        lo, hi = min(n, r * C), min(n, (r + 1) * C)
+        want = root[lo:hi] if r == 0 else bc[min(1, P - 1)][lo:hi]
+        assert sc[r, : hi - lo].tobytes() == want.tobytes()
+        # chunk_bytes are the sizes of the individually compressed chunks
+        assert cb[r] == ccz.compress(root[lo:hi], eb).size
+
+
+def test_chunk_rule():
+    assert ccz.chunk_len(25557032, 16) == 1597440
+    assert ccz.chunk_len(16777216, 8) == 2097152
+    assert ccz.chunk_len(1000, 3) == 384
+    assert ccz.chunk_len(100, 8) == 128     # later chunks are empty

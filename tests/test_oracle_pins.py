@@ -1,0 +1,289 @@
+"""Pins for the oracle (CPU only): everything here checks oracle/ against something other than itself —
+hand-worked streams, invariants the paper fixes, closed forms, identity special cases, brute force."""
+import os
+import struct
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ccz
+from paper_2304_03890_b200 import fields
+from tests import bruteforce_ccz as bf
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+FLT_MIN = np.float32(1.17549435e-38)
+
+
+def load_fixture(name):
+    d, key = {}, None
+    for line in open(os.path.join(GOLDEN, name)):
+        line = line.rstrip("\n")
+        if line.startswith("#") or not line.strip():
+            continue
+        if not line.startswith(" ") and ":" in line:
+            key, val = line.split(":", 1)
+            d[key] = val.strip()
+        else:
+            d[key] += " " + line.strip()
+    return {
+        "L": int(d["block_len"]), "eb": np.float32(d["eb"]),
+        "x": np.array(d["x"].split(), dtype=np.float32),
+        "decoded": np.array(d["decoded"].split(), dtype=np.float32),
+        "stream": np.frombuffer(bytes.fromhex(d["stream"].replace(" ", "")), dtype=np.uint8),
+    }
+
+
+def small_cases():
+    """(name, x, eb) at sizes the oracle finishes in a moment, covering ragged tails and several groups."""
+    rng = np.random.default_rng(7)
+    c1 = fields.config1(n=40000 + 77)
+    c2 = fields.config2(shape=(32, 32, 48), sigma=4.0)
+    c3 = fields.config3(P=1, shape=(32, 32, 32), sigma=4.0)
+    c4 = fields.config4(P=1, shape=(32, 32, 40), sigma=3.0)
+    c5 = fields.config5(P=1, n=33333)
+    out = [("c1", c1["x"].numpy(), c1["eb"]), ("c2", c2["x"].numpy(), c2["eb"]),
+           ("c3", c3["x"][0].numpy(), c3["eb"]), ("c4", c4["x"].numpy(), c4["eb"]),
+           ("c5", c5["x"][0].numpy(), c5["eb"])]
+    out.append(("walk", np.cumsum(rng.normal(0, 0.01, 9000)).astype(np.float32), 1e-3))
+    out.append(("noise", rng.normal(0, 1, 5000).astype(np.float32), 1e-2))
+    out.append(("mixedscale", (rng.normal(0, 1, 6000) * 10.0 ** rng.integers(-6, 3, 6000)).astype(np.float32), 1e-4))
+    return out
+
+
+# ---- hand-worked streams (tests/golden) ----------------------------------------------------------------
+
+@pytest.mark.parametrize("name", ["worked_example_truncated.txt", "worked_example_mixed.txt"])
+def test_hand_worked_stream(name):
+    fx = load_fixture(name)
+    s = ccz.compress(fx["x"], fx["eb"], fx["L"])
+    assert s.tobytes().hex() == fx["stream"].tobytes().hex()
+    for seq in (False, True):
+        d = ccz.decompress(fx["stream"], fx["x"].size, fx["L"], sequential=seq)
+        assert d.tobytes() == fx["decoded"].tobytes()
+    assert np.all(np.abs(fx["decoded"].astype(np.float64)[np.isfinite(fx["x"])]
+                         - fx["x"].astype(np.float64)[np.isfinite(fx["x"])]) <= float(fx["eb"]))
+
+
+# ---- the error bound (Sec. III-B: a chunk compressed once stays within the bound) -----------------------
+
+@pytest.mark.parametrize("case", small_cases(), ids=lambda c: c[0])
+def test_error_bound_and_closed_form(case):
+    _, x, eb = case
+    eb = np.float32(eb)
+    s = ccz.compress(x, eb)
+    d = ccz.decompress(s, x.size)
+    xhat, types = ccz.quantise_only(x, eb)
+    # decoder == stream-free closed form of the quantiser, bit for bit; both decoders agree
+    assert d.tobytes() == xhat.tobytes()
+    assert ccz.decompress(s, x.size, sequential=True).tobytes() == d.tobytes()
+    err = np.abs(d.astype(np.float64) - x.astype(np.float64))
+    assert err.max() <= float(eb) * (1 + 2.0 ** -22)
+    # guard-bit consequence: truncated blocks err by less than eb/2 plus two fp32 roundings
+    t = np.repeat(types, 128)[: x.size]
+    trunc = t == ccz.BLOCK_TRUNCATED
+    if trunc.any():
+        assert err[trunc].max() < float(eb) / 2 + 2.0 ** -22 * np.abs(x).max()
+    assert np.array_equal(d[t == ccz.BLOCK_LOSSLESS], x[t == ccz.BLOCK_LOSSLESS])
+    # the bitmap in the stream says the same as the closed form
+    G = (types.size + 31) // 32
+    bitmap = np.frombuffer(s[32 + 4 * (G + 1): 32 + 4 * (G + 1) + 4 * G].tobytes(), dtype="<u4")
+    bits = ((bitmap[:, None] >> np.arange(32)[None, :]) & 1).reshape(-1)[: types.size]
+    assert np.array_equal(bits, (types != ccz.BLOCK_CONSTANT).astype(bits.dtype))
+
+
+def test_error_bound_fuzz():
+    rng = np.random.default_rng(11)
+    for trial in range(60):
+        n = int(rng.integers(1, 3000))
+        eb = np.float32(10.0 ** rng.uniform(-6, 1))
+        scale = float(eb) * 10.0 ** rng.uniform(-1, 5.5)   # keeps max|x| <= 2^21 eb
+        kind = trial % 3
+        if kind == 0:
+            x = rng.normal(0, scale, n)
+        elif kind == 1:
+            x = np.cumsum(rng.normal(0, scale / 50, n))
+        else:
+            x = rng.uniform(-scale, scale, n) * (rng.random(n) < 0.7)
+        x = x.astype(np.float32)
+        L = int(rng.choice([4, 32, 128, 256]))
+        d = ccz.decompress(ccz.compress(x, eb, L), n, L)
+        assert np.abs(d.astype(np.float64) - x.astype(np.float64)).max() <= float(eb)
+
+
+# ---- constant blocks ---------------------------------------------------------------------------------------
+
+def test_constant_blocks_reproduce_representative():
+    c2 = fields.config2(shape=(32, 32, 48), sigma=4.0)
+    x, eb = c2["x"].numpy(), np.float32(c2["eb"])
+    s = ccz.compress(x, eb)
+    d = ccz.decompress(s, x.size)
+    _, types = ccz.quantise_only(x, eb)
+    xb, db = x.reshape(-1, 128), d.reshape(-1, 128)
+    forced = (xb == xb[:, :1]).all(axis=1)
+    assert forced.mean() > 0.15
+    # every forced block is flagged constant and comes back exactly
+    assert np.all(types[forced] == ccz.BLOCK_CONSTANT)
+    assert np.array_equal(db[forced], xb[forced])
+    assert (types == ccz.BLOCK_CONSTANT).mean() >= forced.mean()
+    # every value of a constant block is one and the same bit pattern: the stored mid-range value
+    const = types == ccz.BLOCK_CONSTANT
+    assert np.all(db[const].view(np.uint32) == db[const][:, :1].view(np.uint32))
+    mid = (np.float32(0.5) * xb[const].min(1) + np.float32(0.5) * xb[const].max(1)).astype(np.float32)
+    assert np.array_equal(db[const][:, 0], mid)
+
+
+def test_identical_values_round_trip_exactly():
+    for c in (3.25, -7.0e-12, 1.0e30, 0.0):
+        x = np.full(300, c, dtype=np.float32)
+        d = ccz.decompress(ccz.compress(x, np.float32(1e-3)), 300)
+        assert d.tobytes() == x.tobytes()
+
+
+def test_gradient_zeros_do_not_make_constant_blocks():
+    c5 = fields.config5(P=1, n=128 * 400)
+    _, types = ccz.quantise_only(c5["x"][0].numpy(), np.float32(c5["eb"]))
+    assert (types == ccz.BLOCK_CONSTANT).mean() < 0.01
+
+
+# ---- lossless path = identity -------------------------------------------------------------------------------
+
+def test_lossless_identity_cases():
+    rng = np.random.default_rng(3)
+    x = rng.normal(0, 1, 1000).astype(np.float32)
+    eb = np.float32(2) * FLT_MIN
+    d = ccz.decompress(ccz.compress(x, eb), x.size)
+    assert d.tobytes() == x.tobytes()
+    # NaN (with payload), +-Inf, -0 inside otherwise ordinary blocks
+    y = rng.normal(0, 1, 512).astype(np.float32)
+    y[5] = np.frombuffer(struct.pack("<I", 0x7FC12345), dtype=np.float32)[0]
+    y[130] = np.inf
+    y[131] = -0.0
+    y[300] = -np.inf
+    y[301] = np.frombuffer(struct.pack("<I", 0xFF800001), dtype=np.float32)[0]
+    xhat, types = ccz.quantise_only(y, np.float32(0.05))
+    assert list(types) == [ccz.BLOCK_LOSSLESS, ccz.BLOCK_LOSSLESS, ccz.BLOCK_LOSSLESS, ccz.BLOCK_TRUNCATED]
+    d = ccz.decompress(ccz.compress(y, np.float32(0.05)), y.size)
+    assert d[:384].tobytes() == y[:384].tobytes()
+    # a block of zeros of both signs is constant and decodes to +0
+    z = np.zeros(128, dtype=np.float32)
+    z[::2] = -0.0
+    d = ccz.decompress(ccz.compress(z, np.float32(1e-3)), 128)
+    assert d.tobytes() == np.zeros(128, dtype=np.float32).tobytes()
+
+
+# ---- closed-form sizes --------------------------------------------------------------------------------------
+
+def test_stream_sizes_closed_form():
+    assert ccz.compress(np.zeros(0, np.float32), np.float32(1.0)).size == 48
+    for G in (1, 2, 5, 33):
+        x = np.full(4096 * G, 2.5, dtype=np.float32)
+        s = ccz.compress(x, np.float32(0.1))
+        front = (36 + 8 * G + 15) // 16 * 16
+        assert s.size == front + 128 * G
+        assert struct.unpack("<Q", s[24:32].tobytes())[0] == s.size
+    # compression-ratio ceiling for L = 128 (the paper's Table II tops out near 124 for SZx)
+    G = 4096
+    s = ccz.compress(np.zeros(4096 * G, np.float32), np.float32(0.1))
+    assert abs(4 * 4096 * G / s.size - 120.47) < 0.05
+    # the worst case meets the bound formula: alternating-sign lossless data, no shared leading bytes
+    n = 4096 * 3 + 130
+    x = np.frombuffer(np.random.default_rng(5).integers(0, 2 ** 32, n, dtype=np.uint32).tobytes(), dtype=np.float32)
+    s = ccz.compress(x, FLT_MIN)
+    assert s.size <= ccz.compress_bound(n)
+    assert ccz.compress_bound(n) == 32 + 4 * 5 + 4 * 4 + 15 + 4 * (64 + 32 * 549 + 3)
+
+
+def test_general_size_formula_from_block_types():
+    """total = front + sum over groups of pad4(2k + 4*const + sum of non-constant record sizes), with the
+    record size of a truncated block derived here from the decoded codes rather than from the stream."""
+    _, x, eb = small_cases()[1]
+    eb = np.float32(eb)
+    s = ccz.compress(x, eb)
+    xhat, types = ccz.quantise_only(x, eb)
+    nb = types.size
+    G = (nb + 31) // 32
+    total = (36 + 8 * G + 15) // 16 * 16
+    for g in range(G):
+        body = 0
+        for b in range(32 * g, min(nb, 32 * g + 32)):
+            blk = x[128 * b: 128 * b + 128]
+            if types[b] == ccz.BLOCK_CONSTANT:
+                body += 4
+                continue
+            _, rec, _ = bf.block_record([np.float32(v) for v in blk], eb)
+            body += 2 + len(rec) // 2
+        total += (body + 3) // 4 * 4
+    assert total == s.size
+
+
+# ---- brute force on tiny inputs -----------------------------------------------------------------------------
+
+def test_bruteforce_tiny_streams():
+    rng = np.random.default_rng(21)
+    for trial in range(40):
+        L = int(rng.choice([4, 8, 32]))
+        n = int(rng.integers(0, 40 * L))
+        eb = np.float32(10.0 ** rng.uniform(-4, 0))
+        x = np.cumsum(rng.normal(0, float(eb) * 10.0 ** rng.uniform(-1, 3), n)).astype(np.float32)
+        if n and trial % 4 == 0:
+            x[rng.integers(0, n)] = np.inf
+        if n > L and trial % 5 == 0:
+            x[:L] = x[0]
+        ref_stream, ref_dec = bf.encode(x, eb, L)
+        s = ccz.compress(x, eb, L)
+        assert s.tobytes() == ref_stream
+        d = ccz.decompress(s, n, L)
+        assert d.tobytes() == np.array(ref_dec, dtype=np.float32).tobytes()
+
+
+def test_two_byte_fields_every_lead_code():
+    """Exhaustive for B = 2: blocks with mu = 0 whose codes are chosen directly, all (prev, cur) pairs of a
+    small alphabet, so that lead 0, 1 and 2 all occur; expected bytes are written out here."""
+    eb = np.float32(0.1875)        # E = 124; with r = 1: m_bits 4, R 13, B 2, q = bits(x) >> 19
+    alphabet = [1.0, -1.0, 0.5, 0.53125, 0.5625, -0.5, 0.25, 1.0 / 64, 0.0]
+    seen = set()
+    for a in alphabet:
+        for b in alphabet:
+            x = np.array([1.0, -1.0, a, b], dtype=np.float32)   # min -1, max 1 -> mu 0, r 1
+            q = [(int(v.view(np.uint32)) >> 19) for v in x]
+            exp_codes, exp_bytes, prev = 0, b"", 0
+            for i, cur in enumerate(q):
+                hi_same = (cur >> 8) == (prev >> 8)
+                lead = 2 if cur == prev else (1 if hi_same else 0)
+                if i >= 2:
+                    seen.add(lead)
+                exp_codes |= lead << (2 * i)
+                exp_bytes += bytes([cur >> 8, cur & 0xFF][lead:])
+                prev = cur
+            s = ccz.compress(x, eb, 4)
+            record = s[48 + 2:].tobytes()
+            expect = struct.pack("<fBB", 0.0, 13, exp_codes) + exp_bytes
+            assert record[: len(expect)] == expect
+            assert all(v == 0 for v in record[len(expect):]) and len(record) - len(expect) < 4
+    assert seen == {0, 1, 2}
+
+
+# ---- corrupt streams are rejected, never read out of bounds --------------------------------------------------
+
+def test_corrupt_streams_are_rejected():
+    _, x, eb = small_cases()[0]
+    s = ccz.compress(x, np.float32(eb))
+    n = x.size
+
+    def bad(stream, n_=n):
+        for seq in (False, True):
+            with pytest.raises(ccz.OracleError) as e:
+                ccz.decompress(stream, n_, sequential=seq)
+            assert e.value.code == ccz.ERR_CORRUPT
+
+    t = s.copy(); t[0] ^= 1; bad(t)                       # magic
+    bad(s[:-4])                                           # truncated
+    bad(s[:20])
+    bad(s, n + 1)                                         # wrong n
+    t = s.copy(); t[36] += 1; bad(t)                      # directory entry moved
+    t = s.copy(); t[24:32] = np.frombuffer(struct.pack("<Q", 2 ** 40), np.uint8); bad(t)
+    G = (n + 4095) // 4096
+    base = (36 + 8 * G + 15) // 16 * 16
+    t = s.copy(); t[base] ^= 0x40; bad(t)                 # first record size wrong
+    t = s.copy(); t[32 + 4 * (G + 1)] ^= 1; bad(t)        # bitmap bit flipped
