@@ -1,0 +1,139 @@
+/*
+ * ccoll.h — C ABI of libccoll: the data-parallel hot path of C-Coll (arXiv 2304.03890) on one B200.
+ *
+ * The library implements, as hand-written sm_100a CUDA kernels,
+ *   - the error-bounded (absolute bound) 1-D fp32 block compressor the paper builds its collectives on
+ *     (Sec. III-C selects the SZx family; Sec. III-E-2 puts the index of variable-length pieces at the
+ *     front of the buffer) and its decoder,
+ *   - the round of the collective-computation framework (Sec. III-A-2, Fig. 4): decompress the received
+ *     chunk, reduce it with the local chunk, recompress — fused, the decoded chunk never reaches HBM,
+ *   - replays of the two frameworks over P virtual ranks that all live in this GPU's memory:
+ *     C-Allreduce = ring reduce-scatter + compressed allgather (Sec. III-E) and C-Bcast / C-Scatter
+ *     (Sec. III-A-1, compress once at the root, decompress once per receiver).  No bytes leave the GPU.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".  The library
+ *     allocates nothing; scratch comes from the workspace the caller registers with ccoll_set_workspace.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is enqueued
+ *     on it and the call returns without waiting.
+ *   - Return value: a ccoll_status_t for errors the host can see (bad argument, missing workspace, CUDA
+ *     launch failure).  Errors only the GPU can see (corrupt stream, capacity, look-back time-out) go to a
+ *     sticky status word in the workspace; read and clear it with ccoll_get_status.
+ *   - Only block_len == 128 is implemented (other values return CCOLL_ERR_UNSUPPORTED).  fp32 buffers must be
+ *     16-byte aligned, streams 16-byte aligned.  n may be any value (ragged last block / group are handled)
+ *     up to CCOLL_MAX_VALUES per stream.
+ *   - Calls that share a workspace must be ordered (same stream, or otherwise serialised by the caller).
+ *
+ * Stream layout "CCZ1" (little endian; nb = ceil(n/128) blocks, G = ceil(nb/32) groups of 32 blocks):
+ *     0 u32 magic 0x315A4343 | 4 u32 flags = 0 | 8 u64 n | 16 u32 block_len | 20 f32 eb | 24 u64 total_bytes
+ *    32 u32 dir[G+1]   start of group g's payload in 4-byte words from payload_base; dir[G] = total words
+ *       u32 bitmap[G]  bit i of word g set iff block 32g+i is not constant
+ *       zero pad to a multiple of 16 -> payload_base
+ *    group payload: u16 record size of every non-constant block (block order), then the records of the
+ *       group's blocks in block order, then zero pad to a multiple of 4.
+ *    record of a constant block: f32 mu.   record of a non-constant block: f32 mu, u8 R, 2-bit lead codes
+ *       (4 per byte, element i at bits 2(i%4)), then for each element its B - lead stored bytes, most
+ *       significant first (B = ceil(R/8)).
+ * Block rules: mu = 0.5*min + 0.5*max; r = max(max - mu, mu - min); r <= eb -> constant.  Otherwise
+ *   R = 10 + E(r) - E(eb) kept bits (sign, exponent, leading mantissa bits) of x - mu, truncated; blocks
+ *   that hold NaN/Inf or would keep 23 or more mantissa bits are stored bit-exactly (R = 32).
+ */
+#ifndef CCOLL_H
+#define CCOLL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CCOLL_OK = 0,
+  CCOLL_ERR_INVALID_ARG = 1, /* null / misaligned pointer, eb not a positive normal float, P < 1, ...       */
+  CCOLL_ERR_UNSUPPORTED = 2, /* block_len != 128, n > CCOLL_MAX_VALUES                                        */
+  CCOLL_ERR_CAPACITY = 3,    /* output stream buffer or workspace too small                                   */
+  CCOLL_ERR_CORRUPT = 4,     /* input stream failed validation; nothing was written for the bad group         */
+  CCOLL_ERR_TIMEOUT = 5,     /* a bounded wait inside a kernel gave up (the kernel still ran to completion)   */
+  CCOLL_ERR_CUDA = 6         /* a CUDA runtime call failed                                                    */
+} ccoll_status_t;
+
+#define CCOLL_BLOCK_LEN 128u
+#define CCOLL_MAX_VALUES ((size_t)1 << 29) /* values per stream (2 GiB of fp32) */
+
+enum { CCOLL_BCAST = 0, CCOLL_SCATTER = 1 };
+
+/* Worst-case stream size in bytes for n values (0 if block_len is unsupported).  Output buffers of
+ * ccoll_compress / ccoll_reduce_step must hold this many bytes. */
+size_t ccoll_compress_bound(size_t n, uint32_t block_len);
+
+/* Chunk length, in values, when n values are divided among P ranks (Sec. III-A-2: the chunk is the input
+ * divided by the number of processes), rounded up to whole blocks so every chunk is 512-byte aligned.
+ * Chunk c covers [min(n, c*len), min(n, (c+1)*len)); trailing chunks may be empty. */
+size_t ccoll_chunk_len(size_t n, int P, uint32_t block_len);
+
+/* Workspace size in bytes needed by any call on buffers of up to n values with up to P virtual ranks
+ * (P = 1 for ccoll_compress / ccoll_decompress / ccoll_reduce_step). */
+size_t ccoll_workspace_bytes(size_t n, uint32_t block_len, int P);
+
+/* Registers caller-owned device memory (256-byte aligned) as the workspace of the CURRENT device and
+ * zeroes it (synchronously).  It must stay valid until replaced.  d_ws = NULL unregisters. */
+int ccoll_set_workspace(void* d_ws, size_t bytes);
+
+/* Waits for `stream`, then returns and clears the sticky device-side status of the current device's
+ * workspace (CCOLL_OK if no kernel reported an error since the last call). */
+int ccoll_get_status(void* stream);
+
+/* Compress n fp32 values with absolute error bound abs_err_bound (Sec. III-C, fixed-accuracy mode).
+ *   in         [n] fp32, 16-byte aligned
+ *   out        stream buffer of at least ccoll_compress_bound(n, block_len) bytes, 16-byte aligned
+ *   out_bytes  device-writable u64 (device or mapped pinned memory), nullable; receives the stream length
+ *              once the stream has been written (the same value is in the stream header at offset 24)
+ * Bytes of `out` past *out_bytes are unspecified.  Every |decoded - in| <= abs_err_bound. */
+int ccoll_compress(const float* in, size_t n, float abs_err_bound, uint32_t block_len, void* out,
+                   uint64_t* out_bytes, void* stream);
+
+/* Decompress a stream of n values made by ccoll_compress / ccoll_reduce_step.
+ *   in        stream, 16-byte aligned; in_bytes = bytes available (host value; >= the stream's own length)
+ *   out       [n] fp32, 16-byte aligned
+ * A stream that fails validation raises CCOLL_ERR_CORRUPT in the device status; no group that failed
+ * validation is written and no byte outside [in, in+in_bytes) or [out, out+n) is touched. */
+int ccoll_decompress(const void* in, size_t in_bytes, size_t n, uint32_t block_len, float* out, void* stream);
+
+/* One round of the ring reduce-scatter of the collective-computation framework (Sec. III-A-2, Fig. 4):
+ *   out = compress( decompress(in) + local ), one fp32 round-to-nearest add per element.
+ *   in        received stream (n values); in_bytes as for ccoll_decompress
+ *   local     [n] fp32 local chunk; must not alias `in`
+ *   out       stream buffer (ccoll_compress_bound bytes); must not alias `in`
+ *   sum_out   nullable [n] fp32: also receives the uncompressed sum (used on the last round, whose
+ *             result the chunk's owner keeps); may equal `local` (in place) */
+int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
+                      uint32_t block_len, void* out, uint64_t* out_bytes, float* sum_out, void* stream);
+
+/* C-Allreduce (SUM) replayed over P virtual ranks in one GPU (Sec. III-E; reduce-scatter per Fig. 4, then
+ * the compress-once allgather of Sec. III-E-1).
+ *   in   [P][n] fp32 rank-major;  out  [P][n] fp32 rank-major (must not alias in)
+ * Chunk c (ccoll_chunk_len) starts at rank c, is compressed there, and visits ranks c+1, c+2, ... (mod P);
+ * each visit is one ccoll_reduce_step.  Rank c-1 owns the final sum: it keeps the uncompressed sum and
+ * does not decompress its own stream; every other rank's copy is the decoded final stream.
+ *   bytes_moved  nullable device u64: compressed bytes that would have crossed the network
+ *                (every reduce-scatter hop once, the final stream P-1 times).
+ * Launches: 1 batched compress, P-1 batched fused reduce steps, 1 batched decode.  P = 1 copies in to out. */
+int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                        uint64_t* bytes_moved, void* stream);
+
+/* C-Bcast / C-Scatter replayed over P virtual ranks, root = rank 0 (Sec. III-A-1: the root compresses each
+ * chunk once, the tree forwards compressed bytes, every receiver decompresses once).
+ *   root_in  [n] fp32
+ *   out      rank r's output starts at out + r*out_rank_stride (stride in floats; 0 = all ranks write the
+ *            same buffer, for timing when P*n floats do not fit — its final contents are then unspecified)
+ *   mode     CCOLL_BCAST: every rank receives n values (rank 0: exact copy; others: all P chunks decoded)
+ *            CCOLL_SCATTER: rank r receives chunk r (rank 0: exact copy of chunk 0)
+ *   chunk_bytes  nullable device u64[P]: compressed size of every chunk */
+int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n,
+                    float abs_err_bound, uint32_t block_len, int mode, uint64_t* chunk_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -443,7 +443,13 @@ int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size
   std::vector<float> s(n);
   int rc = ccz_decompress(in, in_bytes, n, L, s.data());
   if (rc != CCZ_OK) return rc;
-  for (size_t i = 0; i < n; ++i) s[i] = s[i] + local[i];
+  for (size_t i = 0; i < n; ++i) {
+    float t = s[i] + local[i];
+    /* IEEE 754 leaves the payload of a NaN result open (and the paper never mentions NaN); so that the
+     * sum is one well-defined bit pattern on every machine, a NaN sum is stored as the quiet NaN 0x7FFFFFFF. */
+    if (t != t) t = float_of(0x7FFFFFFFu);
+    s[i] = t;
+  }
   rc = ccz_compress(s.data(), n, eb, L, out, cap, out_bytes);
   if (rc != CCZ_OK) return rc;
   if (sum_out)

@@ -1,0 +1,199 @@
+"""Thin Python binding of libccoll's C ABI (include/ccoll.h): argument marshalling only.
+
+Every step of the path runs in the CUDA kernels of libccoll.so; torch is used for device memory and
+streams.  There is no CPU fallback: if the library is missing it is built with nvcc, and if that fails the
+import of a function raises.
+"""
+import ctypes
+
+import torch
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CORRUPT, ERR_TIMEOUT, ERR_CUDA = range(7)
+BCAST, SCATTER = 0, 1
+BLOCK_LEN = 128
+_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CAPACITY", 4: "CORRUPT", 5: "TIMEOUT", 6: "CUDA"}
+
+EXPORTS = ("ccoll_compress_bound", "ccoll_chunk_len", "ccoll_workspace_bytes", "ccoll_set_workspace",
+           "ccoll_get_status", "ccoll_compress", "ccoll_decompress", "ccoll_reduce_step", "ccoll_allreduce_sim",
+           "ccoll_bcast_sim")
+
+_lib = None
+
+
+class CcollError(RuntimeError):
+    def __init__(self, code, where):
+        super().__init__(f"{where}: CCOLL_ERR_{_NAMES.get(code, code)}")
+        self.code = code
+
+
+def lib():
+    """Loads (building first if needed) libccoll.so and declares the C signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    L = ctypes.CDLL(_build.build())
+    sz, u32, f32, i32, vp = ctypes.c_size_t, ctypes.c_uint32, ctypes.c_float, ctypes.c_int, ctypes.c_void_p
+    L.ccoll_compress_bound.restype = sz
+    L.ccoll_compress_bound.argtypes = [sz, u32]
+    L.ccoll_chunk_len.restype = sz
+    L.ccoll_chunk_len.argtypes = [sz, i32, u32]
+    L.ccoll_workspace_bytes.restype = sz
+    L.ccoll_workspace_bytes.argtypes = [sz, u32, i32]
+    L.ccoll_set_workspace.restype = i32
+    L.ccoll_set_workspace.argtypes = [vp, sz]
+    L.ccoll_get_status.restype = i32
+    L.ccoll_get_status.argtypes = [vp]
+    L.ccoll_compress.restype = i32
+    L.ccoll_compress.argtypes = [vp, sz, f32, u32, vp, vp, vp]
+    L.ccoll_decompress.restype = i32
+    L.ccoll_decompress.argtypes = [vp, sz, sz, u32, vp, vp]
+    L.ccoll_reduce_step.restype = i32
+    L.ccoll_reduce_step.argtypes = [vp, sz, vp, sz, f32, u32, vp, vp, vp, vp]
+    L.ccoll_allreduce_sim.restype = i32
+    L.ccoll_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp, vp]
+    L.ccoll_bcast_sim.restype = i32
+    L.ccoll_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp, vp]
+    _lib = L
+    return L
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(rc, where):
+    if rc != OK:
+        raise CcollError(rc, where)
+
+
+# ---- the C ABI, name for name ------------------------------------------------------------------------------
+
+def ccoll_compress_bound(n, block_len=BLOCK_LEN):
+    return int(lib().ccoll_compress_bound(n, block_len))
+
+
+def ccoll_chunk_len(n, P, block_len=BLOCK_LEN):
+    return int(lib().ccoll_chunk_len(n, P, block_len))
+
+
+def ccoll_workspace_bytes(n, block_len=BLOCK_LEN, P=1):
+    return int(lib().ccoll_workspace_bytes(n, block_len, P))
+
+
+_workspaces = {}
+
+
+def ccoll_set_workspace(ws):
+    """ws: uint8 CUDA tensor (kept alive here until replaced) or None."""
+    dev = torch.cuda.current_device()
+    if ws is None:
+        _check(lib().ccoll_set_workspace(None, 0), "ccoll_set_workspace")
+        _workspaces.pop(dev, None)
+        return
+    _check(lib().ccoll_set_workspace(_ptr(ws), ws.numel() * ws.element_size()), "ccoll_set_workspace")
+    _workspaces[dev] = ws
+
+
+def ensure_workspace(n, P=1, block_len=BLOCK_LEN):
+    """Allocates (with torch) and registers a workspace large enough for (n, P) if the current one is not."""
+    need = ccoll_workspace_bytes(n, block_len, P)
+    if need == 0:
+        raise CcollError(ERR_UNSUPPORTED, "ccoll_workspace_bytes")
+    cur = _workspaces.get(torch.cuda.current_device())
+    if cur is None or cur.numel() < need:
+        ccoll_set_workspace(None)
+        _workspaces.pop(torch.cuda.current_device(), None)
+        del cur
+        ccoll_set_workspace(torch.empty(need, dtype=torch.uint8, device="cuda"))
+
+
+def ccoll_get_status(stream=None):
+    return int(lib().ccoll_get_status(_stream(stream)))
+
+
+def ccoll_compress(x, eb, out, out_bytes=None, block_len=BLOCK_LEN, stream=None):
+    _check(lib().ccoll_compress(_ptr(x), x.numel(), eb, block_len, _ptr(out), _ptr(out_bytes), _stream(stream)),
+           "ccoll_compress")
+
+
+def ccoll_decompress(stream_buf, in_bytes, n, out, block_len=BLOCK_LEN, stream=None):
+    _check(lib().ccoll_decompress(_ptr(stream_buf), in_bytes, n, block_len, _ptr(out), _stream(stream)),
+           "ccoll_decompress")
+
+
+def ccoll_reduce_step(in_buf, in_bytes, local, eb, out, out_bytes=None, sum_out=None, block_len=BLOCK_LEN,
+                      stream=None):
+    _check(lib().ccoll_reduce_step(_ptr(in_buf), in_bytes, _ptr(local), local.numel(), eb, block_len, _ptr(out),
+                                   _ptr(out_bytes), _ptr(sum_out), _stream(stream)), "ccoll_reduce_step")
+
+
+def ccoll_allreduce_sim(x, out, eb, bytes_moved=None, block_len=BLOCK_LEN, stream=None):
+    P, n = x.shape
+    _check(lib().ccoll_allreduce_sim(_ptr(x), _ptr(out), P, n, eb, block_len, _ptr(bytes_moved), _stream(stream)),
+           "ccoll_allreduce_sim")
+
+
+def ccoll_bcast_sim(root, out, out_rank_stride, P, eb, mode=BCAST, chunk_bytes=None, block_len=BLOCK_LEN,
+                    stream=None):
+    _check(lib().ccoll_bcast_sim(_ptr(root), _ptr(out), out_rank_stride, P, root.numel(), eb, block_len, mode,
+                                 _ptr(chunk_bytes), _stream(stream)), "ccoll_bcast_sim")
+
+
+# ---- conveniences for tests and examples (allocation with torch, still no arithmetic) -----------------------
+
+def compress(x, eb, block_len=BLOCK_LEN):
+    """Returns the stream as a uint8 CUDA tensor trimmed to its length (synchronises to read the length)."""
+    ensure_workspace(x.numel())
+    out = torch.empty(ccoll_compress_bound(x.numel(), block_len), dtype=torch.uint8, device=x.device)
+    nbytes = torch.zeros(1, dtype=torch.int64, device=x.device)
+    ccoll_compress(x, eb, out, nbytes, block_len)
+    _check(ccoll_get_status(), "ccoll_compress (device)")
+    return out[: int(nbytes.item())]
+
+
+def decompress(stream_buf, n, block_len=BLOCK_LEN):
+    ensure_workspace(n)
+    out = torch.empty(n, dtype=torch.float32, device=stream_buf.device)
+    ccoll_decompress(stream_buf, stream_buf.numel(), n, out, block_len)
+    _check(ccoll_get_status(), "ccoll_decompress (device)")
+    return out
+
+
+def reduce_step(stream_buf, local, eb, want_sum=False, block_len=BLOCK_LEN):
+    n = local.numel()
+    ensure_workspace(n)
+    out = torch.empty(ccoll_compress_bound(n, block_len), dtype=torch.uint8, device=local.device)
+    nbytes = torch.zeros(1, dtype=torch.int64, device=local.device)
+    s = torch.empty_like(local) if want_sum else None
+    ccoll_reduce_step(stream_buf, stream_buf.numel(), local, eb, out, nbytes, s, block_len)
+    _check(ccoll_get_status(), "ccoll_reduce_step (device)")
+    out = out[: int(nbytes.item())]
+    return (out, s) if want_sum else out
+
+
+def allreduce_sim(x, eb, block_len=BLOCK_LEN):
+    P, n = x.shape
+    ensure_workspace(n, P)
+    out = torch.empty_like(x)
+    moved = torch.zeros(1, dtype=torch.int64, device=x.device)
+    ccoll_allreduce_sim(x, out, eb, moved, block_len)
+    _check(ccoll_get_status(), "ccoll_allreduce_sim (device)")
+    return out, int(moved.item())
+
+
+def bcast_sim(root, P, eb, mode=BCAST, block_len=BLOCK_LEN):
+    n = root.numel()
+    ensure_workspace(n, P)
+    stride = n if mode == BCAST else ccoll_chunk_len(n, P, block_len)
+    out = torch.zeros((P, stride), dtype=torch.float32, device=root.device)
+    cb = torch.zeros(P, dtype=torch.int64, device=root.device)
+    ccoll_bcast_sim(root, out, stride, P, eb, mode, cb, block_len)
+    _check(ccoll_get_status(), "ccoll_bcast_sim (device)")
+    return out, cb

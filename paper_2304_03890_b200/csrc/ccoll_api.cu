@@ -1,0 +1,350 @@
+// ccoll_api.cu — the C ABI of libccoll (include/ccoll.h): argument checks, workspace bookkeeping and the
+// launch sequences of the two collective replays.  No device memory is allocated here.
+#include "../../include/ccoll.h"
+#include "ccoll_kernels.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+namespace {
+
+using namespace ccoll;
+
+constexpr size_t kMaxJobs = 1024;  // virtual ranks per replay
+// Workspace layout: [status 256 B][per-job stream sizes, 2 x kMaxJobs u64][look-back words][stream buffers]
+constexpr size_t kOffStatus = 0;
+constexpr size_t kOffJobBytes = 256;
+constexpr size_t kOffTiles = kOffJobBytes + 2 * kMaxJobs * sizeof(uint64_t);
+// The look-back region has a FIXED capacity so that no other data is ever written where a later launch
+// will look for (epoch-tagged) look-back words.
+constexpr size_t kTileCap = (CCOLL_MAX_VALUES / kGroupValues) + kMaxJobs;
+constexpr size_t kOffStreams = kOffTiles + kTileCap * sizeof(uint64_t);
+
+struct Workspace {
+  uint8_t* ptr = nullptr;
+  size_t bytes = 0;
+  uint32_t epoch = 0;
+};
+constexpr int kMaxDevices = 64;
+Workspace g_ws[kMaxDevices];
+std::mutex g_mu;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+size_t groups_of(size_t n) { return (((n + kL - 1) / kL) + kGroupBlocks - 1) / kGroupBlocks; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool valid_eb(float eb) {
+  uint32_t u;
+  std::memcpy(&u, &eb, 4);
+  return std::isfinite(eb) && eb > 0.0f && ((u >> 23) & 0xffu) >= 1u;
+}
+int eb_exponent(float eb) {
+  uint32_t u;
+  std::memcpy(&u, &eb, 4);
+  return (int)((u >> 23) & 0xffu);
+}
+
+int current_ws(Workspace** ws) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return CCOLL_ERR_UNSUPPORTED;
+  *ws = &g_ws[dev];
+  if (!(*ws)->ptr || (*ws)->bytes < kOffStreams) return CCOLL_ERR_CAPACITY;
+  return CCOLL_OK;
+}
+
+// Every launch that uses the look-back words gets a fresh epoch; words tagged with an older epoch read as
+// "not written yet".  When the 32-bit counter wraps, the region is cleared once.
+int next_epoch(Workspace* ws, cudaStream_t s, uint32_t* epoch) {
+  if (++ws->epoch == 0u) {
+    if (cudaMemsetAsync(ws->ptr + kOffTiles, 0, kTileCap * sizeof(uint64_t), s) != cudaSuccess) return CCOLL_ERR_CUDA;
+    ws->epoch = 1u;
+  }
+  *epoch = ws->epoch;
+  return CCOLL_OK;
+}
+
+int check_launch() { return cudaGetLastError() == cudaSuccess ? CCOLL_OK : CCOLL_ERR_CUDA; }
+
+int check_common(size_t n, float eb, uint32_t block_len) {
+  if (block_len < 4 || block_len > 1024 || (block_len % 4)) return CCOLL_ERR_INVALID_ARG;
+  if (!valid_eb(eb)) return CCOLL_ERR_INVALID_ARG;
+  if (block_len != CCOLL_BLOCK_LEN) return CCOLL_ERR_UNSUPPORTED;
+  if (n > CCOLL_MAX_VALUES) return CCOLL_ERR_UNSUPPORTED;
+  return CCOLL_OK;
+}
+
+EncodeBatch make_encode(Workspace* ws, uint32_t epoch, float eb) {
+  EncodeBatch b;
+  std::memset(&b, 0, sizeof(b));
+  b.P = 1;
+  b.tile_state = reinterpret_cast<uint64_t*>(ws->ptr + kOffTiles);
+  b.epoch = epoch;
+  b.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+  b.eb = eb;
+  b.eb_exp = eb_exponent(eb);
+  b.moved_mult = 1;
+  return b;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ccoll_compress_bound(size_t n, uint32_t block_len) {
+  if (block_len != CCOLL_BLOCK_LEN) return 0;
+  size_t G = groups_of(n);
+  return kHeaderBytes + 4 * (G + 1) + 4 * G + 15 + G * ((size_t)kMaxGroupBytes + 3);
+}
+
+size_t ccoll_chunk_len(size_t n, int P, uint32_t block_len) {
+  if (P < 1 || block_len < 4 || block_len > 1024 || (block_len % 4)) return 0;
+  size_t per = (n + (size_t)P - 1) / (size_t)P;
+  return (per + block_len - 1) / block_len * block_len;
+}
+
+size_t ccoll_workspace_bytes(size_t n, uint32_t block_len, int P) {
+  if (block_len != CCOLL_BLOCK_LEN || P < 1 || (size_t)P > kMaxJobs) return 0;
+  if (P == 1) return kOffStreams;
+  size_t C = ccoll_chunk_len(n, P, block_len);
+  return kOffStreams + 2 * (size_t)P * align_up(ccoll_compress_bound(C, block_len), 256);
+}
+
+int ccoll_set_workspace(void* d_ws, size_t bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return CCOLL_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (!d_ws) {
+    g_ws[dev] = Workspace();
+    return CCOLL_OK;
+  }
+  if ((reinterpret_cast<uintptr_t>(d_ws) & 255u) || bytes < kOffStreams) return CCOLL_ERR_INVALID_ARG;
+  if (cudaMemset(d_ws, 0, bytes) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return CCOLL_ERR_CUDA;
+  g_ws[dev].ptr = static_cast<uint8_t*>(d_ws);
+  g_ws[dev].bytes = bytes;
+  g_ws[dev].epoch = 0;
+  return CCOLL_OK;
+}
+
+int ccoll_get_status(void* stream) {
+  Workspace* ws;
+  int rc = current_ws(&ws);
+  if (rc != CCOLL_OK) return rc;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return CCOLL_ERR_CUDA;
+  uint32_t st = 0;
+  if (cudaMemcpy(&st, ws->ptr + kOffStatus, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (st != 0 && cudaMemset(ws->ptr + kOffStatus, 0, 4) != cudaSuccess) return CCOLL_ERR_CUDA;
+  return (int)st;
+}
+
+int ccoll_compress(const float* in, size_t n, float abs_err_bound, uint32_t block_len, void* out, uint64_t* out_bytes,
+                   void* stream) {
+  int rc = check_common(n, abs_err_bound, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (!out || (!in && n) || !aligned16(in) || !aligned16(out) || (reinterpret_cast<uintptr_t>(out_bytes) & 7u))
+    return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint32_t epoch;
+  if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+  EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+  b.x = in;
+  b.chunk_len = n ? n : 1;
+  b.n = n;
+  b.sout = static_cast<uint8_t*>(out);
+  b.out_cap = ccoll_compress_bound(n, block_len);
+  b.out_bytes = out_bytes;
+  size_t G = groups_of(n);
+  b.tiles_per_job = (uint32_t)G;
+  launch_compress(b, (uint32_t)(G ? G : 1), 1, s);
+  return check_launch();
+}
+
+int ccoll_decompress(const void* in, size_t in_bytes, size_t n, uint32_t block_len, float* out, void* stream) {
+  int rc = check_common(n, 1.0f, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (!in || (!out && n) || !aligned16(in) || !aligned16(out)) return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  if (n == 0) return CCOLL_OK;
+  DecodeBatch d;
+  std::memset(&d, 0, sizeof(d));
+  d.sin = static_cast<const uint8_t*>(in);
+  d.sin_bytes_host = in_bytes;
+  d.out = out;
+  d.chunk_len = n;
+  d.n = n;
+  d.P = 1;
+  d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+  launch_decode(d, (uint32_t)groups_of(n), 1, 1, static_cast<cudaStream_t>(stream));
+  return check_launch();
+}
+
+int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
+                      uint32_t block_len, void* out, uint64_t* out_bytes, float* sum_out, void* stream) {
+  int rc = check_common(n, abs_err_bound, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (!in || !out || (!local && n) || !aligned16(in) || !aligned16(out) || !aligned16(local) || !aligned16(sum_out) ||
+      (reinterpret_cast<uintptr_t>(out_bytes) & 7u) || in == out || in == (const void*)local)
+    return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint32_t epoch;
+  if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+  EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+  b.x = local;
+  b.chunk_len = n ? n : 1;
+  b.n = n;
+  b.sin = static_cast<const uint8_t*>(in);
+  b.sin_bytes_host = in_bytes;
+  b.sout = static_cast<uint8_t*>(out);
+  b.out_cap = ccoll_compress_bound(n, block_len);
+  b.out_bytes = out_bytes;
+  b.sum_out = sum_out;
+  size_t G = groups_of(n);
+  b.tiles_per_job = (uint32_t)G;
+  launch_reduce(b, (uint32_t)(G ? G : 1), 1, s);
+  return check_launch();
+}
+
+int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                        uint64_t* bytes_moved, void* stream) {
+  if (P < 1 || (size_t)P > kMaxJobs) return CCOLL_ERR_INVALID_ARG;
+  size_t C = ccoll_chunk_len(n, P, block_len);
+  int rc = check_common(C, abs_err_bound, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (((!in || !out) && n) || !aligned16(in) || !aligned16(out) || (n % 4 && P > 1) || in == out ||
+      (reinterpret_cast<uintptr_t>(bytes_moved) & 7u))
+    return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (bytes_moved && cudaMemsetAsync(bytes_moved, 0, 8, s) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (P == 1) {  // a single rank keeps its data; nothing is compressed or sent
+    if (n && cudaMemcpyAsync(out, in, 4 * n, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CCOLL_ERR_CUDA;
+    return CCOLL_OK;
+  }
+  const size_t S = align_up(ccoll_compress_bound(C, block_len), 256);
+  if (ws->bytes < kOffStreams + 2 * (size_t)P * S) return CCOLL_ERR_CAPACITY;
+  const size_t Gc = groups_of(C);
+  uint8_t* buf[2] = {ws->ptr + kOffStreams, ws->ptr + kOffStreams + (size_t)P * S};
+  uint64_t* bytes[2] = {reinterpret_cast<uint64_t*>(ws->ptr + kOffJobBytes),
+                        reinterpret_cast<uint64_t*>(ws->ptr + kOffJobBytes) + kMaxJobs};
+  const uint32_t gx = (uint32_t)(Gc ? Gc : 1);
+  int cur = 0;
+  for (int k = 0; k < P; ++k) {
+    uint32_t epoch;
+    if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+    EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+    b.x = in;
+    b.x_rank_stride = n;
+    b.chunk_len = C;
+    b.n = n;
+    b.P = P;
+    b.rot = k;  // in round k, chunk c is at rank (c + k) mod P
+    b.s_stride = S;
+    b.out_cap = S;
+    b.moved = bytes_moved;
+    b.moved_mult = (k == P - 1) ? (uint32_t)(P - 1) : 1u;
+    b.tiles_per_job = (uint32_t)Gc;
+    if (k == 0) {
+      b.sout = buf[cur];
+      b.out_bytes = bytes[cur];
+      launch_compress(b, gx, (uint32_t)P, s);
+    } else {
+      b.sin = buf[cur];
+      b.sin_bytes = bytes[cur];
+      b.sout = buf[cur ^ 1];
+      b.out_bytes = bytes[cur ^ 1];
+      if (k == P - 1) {  // the owner keeps the uncompressed sum
+        b.sum_out = out;
+        b.sum_rank_stride = n;
+      }
+      launch_reduce(b, gx, (uint32_t)P, s);
+      cur ^= 1;
+    }
+    if ((rc = check_launch()) != CCOLL_OK) return rc;
+  }
+  // allgather: every rank but the owner decodes the final stream of every chunk
+  DecodeBatch d;
+  std::memset(&d, 0, sizeof(d));
+  d.sin = buf[cur];
+  d.s_stride = S;
+  d.sin_bytes = bytes[cur];
+  d.out = out;
+  d.out_rank_stride = n;
+  d.chunk_len = C;
+  d.n = n;
+  d.P = P;
+  d.skip_mode = 1;
+  d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+  if (Gc) launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s);
+  return check_launch();
+}
+
+int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float abs_err_bound,
+                    uint32_t block_len, int mode, uint64_t* chunk_bytes, void* stream) {
+  if (P < 1 || (size_t)P > kMaxJobs || (mode != CCOLL_BCAST && mode != CCOLL_SCATTER)) return CCOLL_ERR_INVALID_ARG;
+  size_t C = ccoll_chunk_len(n, P, block_len);
+  int rc = check_common(C, abs_err_bound, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (((!root_in || !out) && n) || !aligned16(root_in) || !aligned16(out) || (out_rank_stride % 4) ||
+      (reinterpret_cast<uintptr_t>(chunk_bytes) & 7u))
+    return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  const size_t S = align_up(ccoll_compress_bound(C, block_len), 256);
+  if (ws->bytes < kOffStreams + (size_t)P * S) return CCOLL_ERR_CAPACITY;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t Gc = groups_of(C);
+  uint8_t* buf = ws->ptr + kOffStreams;
+  uint64_t* bytes = reinterpret_cast<uint64_t*>(ws->ptr + kOffJobBytes);
+  // the root compresses every chunk exactly once
+  uint32_t epoch;
+  if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+  EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+  b.x = root_in;
+  b.chunk_len = C;
+  b.n = n;
+  b.P = P;
+  b.sout = buf;
+  b.s_stride = S;
+  b.out_cap = S;
+  b.out_bytes = bytes;
+  b.tiles_per_job = (uint32_t)Gc;
+  launch_compress(b, (uint32_t)(Gc ? Gc : 1), (uint32_t)P, s);
+  if ((rc = check_launch()) != CCOLL_OK) return rc;
+  if (chunk_bytes &&
+      cudaMemcpyAsync(chunk_bytes, bytes, (size_t)P * sizeof(uint64_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return CCOLL_ERR_CUDA;
+  // the root keeps its own data uncompressed
+  size_t own = (mode == CCOLL_BCAST) ? n : (C < n ? C : n);
+  if (own && cudaMemcpyAsync(out, root_in, 4 * own, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CCOLL_ERR_CUDA;
+  if (P == 1 || Gc == 0) return CCOLL_OK;
+  DecodeBatch d;
+  std::memset(&d, 0, sizeof(d));
+  d.sin = buf;
+  d.s_stride = S;
+  d.sin_bytes = bytes;
+  d.out = out;
+  d.out_rank_stride = out_rank_stride;
+  d.chunk_len = C;
+  d.n = n;
+  d.P = P;
+  d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+  if (mode == CCOLL_BCAST) {
+    d.skip_mode = 2;  // rank 0 is the root
+    launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s);
+  } else {
+    d.skip_mode = 3;  // chunk 0 stays at the root
+    d.scatter = 1;
+    launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s);
+  }
+  return check_launch();
+}
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// ccoll_kernels.cuh — sm_100a kernels of the C-Coll hot path: block classify + encode + size scan and
+// compaction (compress), the parallel decoder, and the fused decompress-add-recompress ring round.
+//
+// Work decomposition (all three kernels): one CTA of 4 warps owns one GROUP of 32 blocks (4096 values);
+// warp w owns blocks 8w .. 8w+7 of it; within a block lane l owns elements 4l .. 4l+3, i.e. exactly one
+// 128-bit coalesced load / store.  Everything a block needs from its neighbours' lanes travels by warp
+// shuffles or warp reductions; the variable-length bytes are assembled in registers, placed into a
+// shared-memory image of the group's payload, and leave the SM as coalesced word stores at the offset
+// found by a decoupled look-back over the groups' sizes.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace ccoll {
+
+constexpr uint32_t kMagic = 0x315A4343u;  // "CCZ1"
+constexpr int kL = 128;                    // values per block
+constexpr int kGroupBlocks = 32;           // blocks per group
+constexpr int kGroupValues = kL * kGroupBlocks;
+constexpr int kWarps = 4;
+constexpr int kThreads = 32 * kWarps;
+constexpr int kWarpBlocks = kGroupBlocks / kWarps;  // 8 blocks per warp
+constexpr int kHeaderBytes = 32;
+constexpr int kMaxRecord = 5 + kL / 4 + 4 * kL;                       // 549
+constexpr int kMaxGroupBytes = 2 * kGroupBlocks + kGroupBlocks * kMaxRecord;  // 17632 (a multiple of 4)
+constexpr int kImgWords = kMaxGroupBytes / 4 + 24;                    // image + slack for 5-word windows
+
+// status codes mirrored from ccoll.h
+constexpr uint32_t kErrCapacity = 3, kErrCorrupt = 4, kErrTimeout = 5;
+
+// Look-back state word: [epoch:32][flag:2][value:30].  A word whose epoch differs from the launch's epoch
+// is "not written yet", so the state array never needs clearing between launches.
+constexpr uint32_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
+constexpr uint32_t kValueMask = (1u << 30) - 1;
+constexpr uint32_t kSpinLimit = 1u << 21;  // polls (each followed by a short sleep) before giving up
+
+// A family of encode jobs (one job per blockIdx.y): job y covers values [y*C, min(n, (y+1)*C)) of the
+// buffer of virtual rank (y + rot) mod P.
+struct EncodeBatch {
+  const float* x;           // fp32 inputs: the data to compress, or the local chunk of a reduce step
+  uint64_t x_rank_stride;   // floats between ranks
+  uint64_t chunk_len;       // C
+  uint64_t n;               // values per rank buffer
+  int P, rot;
+  const uint8_t* sin;       // incoming streams (reduce step only), job y at sin + y*s_stride
+  const uint64_t* sin_bytes;  // device array indexed by job, or null -> sin_bytes_host
+  uint64_t sin_bytes_host;
+  uint8_t* sout;            // outgoing streams, job y at sout + y*s_stride
+  uint64_t s_stride;
+  uint64_t out_cap;         // bytes available per outgoing stream
+  uint64_t* out_bytes;      // device array indexed by job (nullable)
+  float* sum_out;           // nullable; addressed like x (rank (y+rot) mod P, chunk y) with sum_rank_stride
+  uint64_t sum_rank_stride;
+  uint64_t* moved;          // nullable: += moved_mult * stream bytes of every job
+  uint32_t moved_mult;
+  uint64_t* tile_state;     // look-back words, job y at tile_state + y*tiles_per_job
+  uint32_t tiles_per_job;
+  uint32_t epoch;
+  uint32_t* status;         // sticky error word
+  float eb;
+  int eb_exp;               // biased exponent field of eb
+};
+
+// A family of decode jobs: blockIdx.y = stream (chunk) index, blockIdx.z = destination rank.
+struct DecodeBatch {
+  const uint8_t* sin;
+  uint64_t s_stride;
+  const uint64_t* sin_bytes;
+  uint64_t sin_bytes_host;
+  float* out;
+  uint64_t out_rank_stride;  // floats between destination ranks
+  uint64_t chunk_len;
+  uint64_t n;
+  int P;
+  int skip_mode;   // 0 none; 1 skip rank z == (y-1) mod P (the chunk's owner); 2 skip z == 0; 3 skip y == 0
+  int scatter;     // 1: job y writes at out + y*out_rank_stride; 0: at out + z*out_rank_stride + y*C
+  uint32_t* status;
+};
+
+void launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
+void launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
+void launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s);
+
+}  // namespace ccoll

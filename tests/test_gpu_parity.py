@@ -1,0 +1,243 @@
+"""Parity of the CUDA path (through the C ABI) with the oracle: stream bytes, block flags and decoded values
+must be bit-identical; the collective replays must match the oracle's identical ring order bit for bit."""
+import struct
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ccz
+from paper_2304_03890_b200 import binding as B
+from paper_2304_03890_b200 import fields
+
+pytestmark = pytest.mark.gpu
+FLT_MIN = np.float32(1.17549435e-38)
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def check_codec(x, eb):
+    """compress / decompress on the GPU vs the oracle, byte for byte."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    eb = float(np.float32(eb))
+    ref = ccz.compress(x, eb)
+    got = B.compress(dev(x), eb)
+    g = got.cpu().numpy()
+    assert g.size == ref.size, (g.size, ref.size)
+    if not np.array_equal(g, ref):
+        bad = np.flatnonzero(g != ref)
+        raise AssertionError(f"stream differs at {bad[:8]} of {ref.size}: got {g[bad[:8]]} want {ref[bad[:8]]}")
+    dref = ccz.decompress(ref, x.size)
+    dgot = B.decompress(got, x.size).cpu().numpy()
+    assert dgot.tobytes() == dref.tobytes()
+    return ref
+
+
+EDGE_SIZES = [0, 1, 3, 4, 5, 127, 128, 129, 130, 255, 4095, 4096, 4097, 4096 + 128, 4096 * 3 + 130, 4096 * 8,
+              4096 * 37 + 1000 + 3]
+
+
+@pytest.mark.parametrize("n", EDGE_SIZES)
+def test_edge_sizes(n):
+    rng = np.random.default_rng(n + 1)
+    x = np.cumsum(rng.normal(0, 0.01, n)).astype(np.float32)
+    check_codec(x, 1e-3)
+
+
+def test_special_blocks():
+    rng = np.random.default_rng(3)
+    n = 4096 * 2 + 700
+    x = rng.normal(0, 1, n).astype(np.float32)
+    x[5] = np.frombuffer(struct.pack("<I", 0x7FC12345), dtype=np.float32)[0]   # NaN with payload
+    x[130] = np.inf
+    x[131] = -0.0
+    x[300] = -np.inf
+    x[301] = np.frombuffer(struct.pack("<I", 0xFF800001), dtype=np.float32)[0]  # signalling NaN
+    x[1024:1152] = 0.0
+    x[1024:1152:2] = -0.0                    # zeros of both signs
+    x[2048:2176] = 3.5                       # constant
+    x[4096:4224] = 1e30 * rng.normal(0, 1, 128)   # huge next to small -> wide exponent range
+    x[n - 50:] = np.nan                      # NaNs in the ragged tail block
+    check_codec(x, 0.05)
+    check_codec(x, 2 * FLT_MIN)              # everything lossless
+    check_codec(np.full(5000, 2.5, np.float32), 0.1)   # everything constant
+    check_codec(np.zeros(4096 * 5, np.float32), 1.0)
+    check_codec(rng.normal(0, 1e-30, 3000).astype(np.float32), 1e-3)   # tiny values, constant blocks
+    # random bit patterns: subnormals, NaNs, Infs everywhere
+    bits = rng.integers(0, 2 ** 32, 4096 * 2 + 77, dtype=np.uint32)
+    check_codec(np.frombuffer(bits.tobytes(), dtype=np.float32), 1e-3)
+
+
+def test_power_of_two_bound_and_wide_ranges():
+    rng = np.random.default_rng(9)
+    x = rng.uniform(0, 1000, 4096 * 4 + 9).astype(np.float32)
+    check_codec(x, 1.0)
+    check_codec(x, 0.5)
+    check_codec((rng.normal(0, 1, 9000) * 10.0 ** rng.integers(-6, 3, 9000)).astype(np.float32), 1e-4)
+    for e in range(-12, 6):
+        check_codec(rng.normal(0, 1, 1500).astype(np.float32), 10.0 ** e)
+
+
+def small_configs():
+    c1 = fields.config1(n=1 << 18)
+    c2 = fields.config2(shape=(64, 64, 64), sigma=8.0)
+    c3 = fields.config3(P=1, shape=(64, 64, 32), sigma=4.0)
+    c4 = fields.config4(P=1, shape=(64, 32, 64), sigma=6.0)
+    c5 = fields.config5(P=1, n=255570 + 32)
+    return [("c1", c1["x"].numpy(), c1["eb"]), ("c2", c2["x"].numpy(), c2["eb"]),
+            ("c3", c3["x"][0].numpy(), c3["eb"]), ("c4", c4["x"].numpy(), c4["eb"]),
+            ("c5", c5["x"][0].numpy(), c5["eb"])]
+
+
+@pytest.mark.parametrize("case", small_configs(), ids=lambda c: c[0])
+def test_config_shaped_inputs(case):
+    _, x, eb = case
+    check_codec(x, eb)
+
+
+def test_config1_full_size():
+    c1 = fields.config1()
+    check_codec(c1["x"].numpy(), c1["eb"])
+
+
+def test_reduce_step_matches_oracle():
+    c = fields.config3(P=3, shape=(32, 32, 40), sigma=3.0)
+    x, eb = c["x"].numpy(), float(np.float32(c["eb"]))
+    for n in (x.shape[1], 4096 * 2 + 130, 129, 1):
+        a, b_, c_ = x[0, :n], x[1, :n], x[2, :n]
+        s0 = ccz.compress(a, eb)
+        ref1, sum1 = ccz.reduce_step(s0, b_, eb, want_sum=True)
+        got1, gsum1 = B.reduce_step(dev(s0), dev(b_), eb, want_sum=True)
+        assert np.array_equal(got1.cpu().numpy(), ref1)
+        assert gsum1.cpu().numpy().tobytes() == sum1.tobytes()
+        # chain a second round from the GPU's own output, without sum_out
+        ref2 = ccz.reduce_step(ref1, c_, eb)
+        got2 = B.reduce_step(got1, dev(c_), eb)
+        assert np.array_equal(got2.cpu().numpy(), ref2)
+
+
+def test_reduce_step_in_place_sum_and_special_values():
+    rng = np.random.default_rng(4)
+    n = 4096 + 300
+    a = rng.normal(0, 1, n).astype(np.float32)
+    b_ = rng.normal(0, 1, n).astype(np.float32)
+    a[7] = np.inf
+    b_[200] = np.nan
+    b_[4096:] = -a[4096:]            # sums to exact zeros -> constant tail
+    eb = 1e-2
+    s0 = ccz.compress(a, eb)
+    ref, rsum = ccz.reduce_step(s0, b_, eb, want_sum=True)
+    local = dev(b_)
+    out = torch.empty(B.ccoll_compress_bound(n), dtype=torch.uint8, device="cuda")
+    nbytes = torch.zeros(1, dtype=torch.int64, device="cuda")
+    B.ensure_workspace(n)
+    B.ccoll_reduce_step(dev(s0), s0.size, local, eb, out, nbytes, local)   # sum_out aliases local
+    assert B.ccoll_get_status() == B.OK
+    assert np.array_equal(out[: int(nbytes.item())].cpu().numpy(), ref)
+    assert local.cpu().numpy().tobytes() == rsum.tobytes()
+
+
+@pytest.mark.parametrize("P,n", [(2, 4096 * 2), (3, 128 * 37 + 4), (4, 4096 * 5 + 1000), (8, 32 * 32 * 40),
+                                 (5, 8), (16, 128 * 16 * 3 + 40)])
+def test_allreduce_sim_matches_oracle(P, n):
+    c = fields.config3(P=P, shape=(32, 32, 40), sigma=3.0)
+    x = np.ascontiguousarray(c["x"].numpy()[:, :n])
+    eb = float(np.float32(c["eb"]))
+    ref, ref_moved = ccz.allreduce_sim(x, eb)
+    got, moved = B.allreduce_sim(dev(x), eb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes()
+    assert moved == ref_moved
+    # and the benchmark spec's bound: within P*eb of the fp64 sum
+    exact = x.astype(np.float64).sum(0)
+    assert np.abs(got.cpu().numpy() - exact[None]).max() <= P * eb + P * 2.0 ** -23 * np.abs(exact).max()
+
+
+def test_allreduce_sim_gradient_shaped():
+    c = fields.config5(P=4, n=128 * 1000 + 40)
+    x, eb = c["x"].numpy(), float(np.float32(c["eb"]))
+    ref, ref_moved = ccz.allreduce_sim(x, eb)
+    got, moved = B.allreduce_sim(dev(x), eb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
+
+
+def test_allreduce_single_rank_is_identity():
+    x = torch.randn(1, 1000, device="cuda")
+    got, moved = B.allreduce_sim(x, 1e-3)
+    assert torch.equal(got, x) and moved == 0
+
+
+@pytest.mark.parametrize("P", [1, 3, 8, 32])
+@pytest.mark.parametrize("mode", [B.BCAST, B.SCATTER])
+def test_bcast_sim_matches_oracle(P, mode):
+    c = fields.config4(P=P, shape=(16, 32, 40), sigma=3.0)
+    root = np.ascontiguousarray(c["x"].numpy()[: 16 * 32 * 40 - 20])
+    eb = float(np.float32(c["eb"]))
+    ref, ref_cb = ccz.bcast_sim(root, P, eb, mode=mode)
+    got, cb = B.bcast_sim(dev(root), P, eb, mode=mode)
+    assert np.array_equal(cb.cpu().numpy().astype(np.uint64), ref_cb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes()
+
+
+def test_corrupt_streams_raise_status_and_write_nothing():
+    c1 = fields.config1(n=4096 * 6 + 100)
+    x, eb = c1["x"].numpy(), float(np.float32(c1["eb"]))
+    n = x.size
+    s = ccz.compress(x, eb)
+    G = (n + 4095) // 4096
+    base = (36 + 8 * G + 15) // 16 * 16
+
+    def run(stream, n_=n):
+        out = torch.full((n_,), -7.0, device="cuda")
+        B.ensure_workspace(n_)
+        B.ccoll_decompress(dev(stream), stream.size, n_, out)
+        return B.ccoll_get_status(), out.cpu().numpy()
+
+    st, out = run(s)
+    assert st == B.OK and out.tobytes() == ccz.decompress(s, n).tobytes()
+    t = s.copy(); t[0] ^= 1
+    st, out = run(t)
+    assert st == B.ERR_CORRUPT and np.all(out == -7.0)
+    st, out = run(s[:-4])
+    assert st == B.ERR_CORRUPT and np.all(out == -7.0)
+    st, out = run(s, n + 1)
+    assert st == B.ERR_CORRUPT and np.all(out == -7.0)
+    t = s.copy(); t[24:32] = np.frombuffer(struct.pack("<Q", 2 ** 40), np.uint8)
+    st, out = run(t)
+    assert st == B.ERR_CORRUPT and np.all(out == -7.0)
+    # damage inside group 2 only: that group is not written, the others are
+    d2 = struct.unpack("<I", s[32 + 8: 32 + 12].tobytes())[0]
+    t = s.copy(); t[base + 4 * d2] ^= 0x40     # first record size of group 2
+    st, out = run(t)
+    assert st == B.ERR_CORRUPT
+    good = ccz.decompress(s, n)
+    assert np.all(out[2 * 4096: 3 * 4096] == -7.0)
+    assert out[: 2 * 4096].tobytes() == good[: 2 * 4096].tobytes()
+    assert out[3 * 4096:].tobytes() == good[3 * 4096:].tobytes()
+    # a lead code larger than the field width (B = 2 here means code 3 is impossible)
+    t = s.copy(); t[32 + 4 * (G + 1)] ^= 1      # flip a bitmap bit -> sizes no longer add up
+    st, out = run(t)
+    assert st == B.ERR_CORRUPT and np.all(out[:4096] == -7.0)
+    # the status is sticky until read, then cleared
+    assert B.ccoll_get_status() == B.OK
+
+
+def test_argument_checks():
+    L = B.lib()
+    B.ensure_workspace(1024)
+    x = torch.zeros(1024, device="cuda")
+    out = torch.empty(B.ccoll_compress_bound(1024), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.CcollError) as e:
+        B.ccoll_compress(x, 0.0, out)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.CcollError) as e:
+        B.ccoll_compress(x, float("nan"), out)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.CcollError) as e:
+        B.ccoll_compress(x, 1e-3, out, block_len=64)
+    assert e.value.code == B.ERR_UNSUPPORTED
+    with pytest.raises(B.CcollError) as e:
+        B.ccoll_compress(x[1:], 1e-3, out)       # misaligned
+    assert e.value.code == B.ERR_INVALID_ARG
+    assert L.ccoll_compress(None, 8, 1e-3, 128, None, None, None) == B.ERR_INVALID_ARG
