@@ -291,17 +291,17 @@ def main():
     peak, peak_kind = measured_peaks()
     S1, S2 = int(nb1.item()), int(nb2.item())
     alg = {
-        "compress_kernel": 4 * n + S1,
-        "decode_kernel": S1 + 4 * n,
-        "reduce_kernel": S1 + 4 * n + S2 + 4 * n,   # stream in + local in + stream out + sum_out
+        "ccoll_compress_kernel": 4 * n + S1,
+        "ccoll_decode_kernel": S1 + 4 * n,
+        "ccoll_reduce_kernel": S1 + 4 * n + S2 + 4 * n,   # stream in + local in + stream out + sum_out
     }
     roofs = {}
-    for name, ms in zip(("compress_kernel", "decode_kernel", "reduce_kernel"), call_ms[:3]):
+    for name, ms in zip(("ccoll_compress_kernel", "ccoll_decode_kernel", "ccoll_reduce_kernel"), call_ms[:3]):
         ach = alg[name] / (ms * 1e-3) / 1e9
         roofs[name] = {"bound": "hbm", "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                        "frac": ach / peak, "traffic": None, "algorithmic_bytes": alg[name], "ms": ms,
                        "input_GBps": 4 * n / (ms * 1e-3) / 1e9}
-    dominant = "reduce_kernel"
+    dominant = "ccoll_reduce_kernel"
     roofline = dict(roofs[dominant], kernel=dominant)
 
     # ---- end to end: inputs from pinned host memory, results read back, all inside the timed region ----

@@ -18,7 +18,7 @@ constexpr size_t kOffJobBytes = 256;
 constexpr size_t kOffTiles = kOffJobBytes + 2 * kMaxJobs * sizeof(uint64_t);
 // The look-back region has a FIXED capacity so that no other data is ever written where a later launch
 // will look for (epoch-tagged) look-back words.
-constexpr size_t kTileCap = (CCOLL_MAX_VALUES / kGroupValues) + kMaxJobs;
+constexpr size_t kTileCap = (CCOLL_MAX_VALUES / kGroupValues) * 33 / 32 + 2 * kMaxJobs;
 constexpr size_t kOffStreams = kOffTiles + kTileCap * sizeof(uint64_t);
 
 struct Workspace {
@@ -159,7 +159,8 @@ int ccoll_compress(const float* in, size_t n, float abs_err_bound, uint32_t bloc
   b.out_bytes = out_bytes;
   size_t G = groups_of(n);
   b.tiles_per_job = (uint32_t)G;
-  launch_compress(b, (uint32_t)(G ? G : 1), 1, s);
+  b.state_stride = (uint32_t)(G + (G + 31) / 32);
+  if (!launch_compress(b, (uint32_t)(G ? G : 1), 1, s)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
 
@@ -179,7 +180,7 @@ int ccoll_decompress(const void* in, size_t in_bytes, size_t n, uint32_t block_l
   d.n = n;
   d.P = 1;
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
-  launch_decode(d, (uint32_t)groups_of(n), 1, 1, static_cast<cudaStream_t>(stream));
+  if (!launch_decode(d, (uint32_t)groups_of(n), 1, 1, static_cast<cudaStream_t>(stream))) return CCOLL_ERR_CUDA;
   return check_launch();
 }
 
@@ -207,7 +208,8 @@ int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_
   b.sum_out = sum_out;
   size_t G = groups_of(n);
   b.tiles_per_job = (uint32_t)G;
-  launch_reduce(b, (uint32_t)(G ? G : 1), 1, s);
+  b.state_stride = (uint32_t)(G + (G + 31) / 32);
+  if (!launch_reduce(b, (uint32_t)(G ? G : 1), 1, s)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
 
@@ -251,10 +253,11 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
     b.moved = bytes_moved;
     b.moved_mult = (k == P - 1) ? (uint32_t)(P - 1) : 1u;
     b.tiles_per_job = (uint32_t)Gc;
+    b.state_stride = (uint32_t)(Gc + (Gc + 31) / 32);
     if (k == 0) {
       b.sout = buf[cur];
       b.out_bytes = bytes[cur];
-      launch_compress(b, gx, (uint32_t)P, s);
+      if (!launch_compress(b, gx, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
     } else {
       b.sin = buf[cur];
       b.sin_bytes = bytes[cur];
@@ -264,7 +267,7 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
         b.sum_out = out;
         b.sum_rank_stride = n;
       }
-      launch_reduce(b, gx, (uint32_t)P, s);
+      if (!launch_reduce(b, gx, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
       cur ^= 1;
     }
     if ((rc = check_launch()) != CCOLL_OK) return rc;
@@ -282,7 +285,7 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
   d.P = P;
   d.skip_mode = 1;
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
-  if (Gc) launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s);
+  if (Gc && !launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
 
@@ -316,7 +319,8 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   b.out_cap = S;
   b.out_bytes = bytes;
   b.tiles_per_job = (uint32_t)Gc;
-  launch_compress(b, (uint32_t)(Gc ? Gc : 1), (uint32_t)P, s);
+  b.state_stride = (uint32_t)(Gc + (Gc + 31) / 32);
+  if (!launch_compress(b, (uint32_t)(Gc ? Gc : 1), (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   if ((rc = check_launch()) != CCOLL_OK) return rc;
   if (chunk_bytes &&
       cudaMemcpyAsync(chunk_bytes, bytes, (size_t)P * sizeof(uint64_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
@@ -338,11 +342,11 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
   if (mode == CCOLL_BCAST) {
     d.skip_mode = 2;  // rank 0 is the root
-    launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s);
+    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   } else {
     d.skip_mode = 3;  // chunk 0 stays at the root
     d.scatter = 1;
-    launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s);
+    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s)) return CCOLL_ERR_CUDA;
   }
   return check_launch();
 }

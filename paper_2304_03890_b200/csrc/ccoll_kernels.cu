@@ -1,12 +1,29 @@
 // ccoll_kernels.cu — device code of libccoll (see ccoll_kernels.cuh for the work decomposition and
 // include/ccoll.h for the stream layout and the block rules).  Compiled with --fmad=false: every fp32
 // operation of the block rules rounds once, exactly as stated.
+//
+// Lane mapping (all kernels): thread tid of the CTA owns SLICE tid of the group = 32 consecutive values
+// (128 bytes); block = tid / 4, so four neighbouring lanes share a block and everything that must cross
+// lanes (min/max, the predecessor code, byte offsets) is a two-step shuffle inside that quad of lanes.
+// Per-value work runs serially inside a lane over eight 128-bit quads, so per-block quantities (mid-range,
+// required bits, header) cost 4 lanes, not 32.
+//
+// Data movement: fp32 values enter and leave through shared-memory rows: warps move 512 contiguous bytes per
+// 128-bit load / store instruction and (un)scatter them into per-lane slices padded to 144 bytes, which
+// keeps both the transposing accesses and the lanes' own 128-bit accesses conflict free.  (One 128-byte
+// bulk-async copy per lane was measured first: a million such copies per 134 MB capped the kernel near
+// 1.2 TB/s, so plain coalesced loads replaced them.)  Variable-length bytes are first appended to the
+// lane's own slice (aligned word stores), then copied once to their byte offset in a shared-memory image
+// of the group's payload, which leaves as coalesced word stores at the offset a decoupled look-back yields.
 #include "ccoll_kernels.cuh"
 
 namespace ccoll {
 namespace {
 
 constexpr uint32_t kFull = 0xffffffffu;
+constexpr int kSliceVals = 32;                      // values per lane
+constexpr int kSliceBytes = 144;                    // 128 data bytes + 16 pad
+constexpr int kRowsBytes = kThreads * kSliceBytes;  // 18432
 
 // ---------------------------------------------------------------------------------------------------
 // small helpers
@@ -21,15 +38,15 @@ __device__ __forceinline__ float min_nan(float a, float b) {
   asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
   return r;
 }
-// Warp-wide fp32 max / min in one instruction; a NaN in any lane makes the result NaN.
-__device__ __forceinline__ float warp_max_nan(float v) {
+// three-input forms (sm_100): fold two new values into a running extreme with one instruction
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
   float r;
-  asm volatile("redux.sync.max.NaN.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-__device__ __forceinline__ float warp_min_nan(float v) {
+__device__ __forceinline__ float min3_nan(float a, float b, float c) {
   float r;
-  asm volatile("redux.sync.min.NaN.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
 __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t* p) {
@@ -44,7 +61,6 @@ __device__ __forceinline__ uint64_t pack_state(uint32_t epoch, uint32_t flag, ui
   return ((uint64_t)epoch << 32) | ((uint64_t)flag << 30) | (uint64_t)(value & kValueMask);
 }
 __device__ __forceinline__ void raise(uint32_t* status, uint32_t code) { atomicMax(status, code); }
-
 __device__ __forceinline__ uint32_t payload_base(uint32_t G) { return (kHeaderBytes + 8u * G + 4u + 15u) & ~15u; }
 
 // unaligned reads from a word image in shared memory
@@ -55,7 +71,26 @@ __device__ __forceinline__ uint32_t img_u32(const uint32_t* img, uint32_t byte_o
 __device__ __forceinline__ uint32_t img_u8(const uint32_t* img, uint32_t byte_off) {
   return (img[byte_off >> 2] >> (8u * (byte_off & 3u))) & 0xffu;
 }
+// The outgoing image is zeroed once and its shared words are filled by atomic OR, so bytes of one word
+// may come from any lane.
+__device__ __forceinline__ void or_u8(uint32_t* img, uint32_t off, uint32_t byte) {
+  atomicOr(&img[off >> 2], (byte & 0xffu) << (8u * (off & 3u)));
+}
+__device__ __forceinline__ void or_u32(uint32_t* img, uint32_t off, uint32_t v) {
+  uint32_t z = 8u * (off & 3u), w = off >> 2;
+  atomicOr(&img[w], v << z);
+  if (z) atomicOr(&img[w + 1], v >> (32u - z));
+}
+__device__ __forceinline__ void or_u64(uint32_t* img, uint32_t off, uint32_t lo, uint32_t hi) {
+  uint32_t z = 8u * (off & 3u), w = off >> 2;
+  atomicOr(&img[w], lo << z);
+  atomicOr(&img[w + 1], __funnelshift_l(lo, hi, z));
+  if (z) atomicOr(&img[w + 2], hi >> (32u - z));
+}
 
+// ---------------------------------------------------------------------------------------------------
+// geometry
+// ---------------------------------------------------------------------------------------------------
 struct JobGeom {
   uint64_t lo;      // first value of the job inside the rank buffer
   uint64_t len;     // values in the job
@@ -74,136 +109,320 @@ __device__ __forceinline__ JobGeom job_geom(uint64_t n, uint64_t C, uint32_t y) 
   j.m_last = (uint32_t)(j.len - (uint64_t)(j.nb ? j.nb - 1 : 0) * kL);
   return j;
 }
+// What a thread owns in group g: its block's value count and its own valid values.
+struct LaneGeom {
+  uint32_t blk;    // block inside the group (tid / 4)
+  uint32_t t;      // slice inside the block (tid % 4)
+  uint32_t m_blk;  // values in the block (0 = the block does not exist)
+  uint32_t nv;     // valid values in this lane's slice (0..32)
+  uint32_t nfull;  // complete slices in the whole group
+  uint64_t first;  // index (inside the job) of the slice's first value
+};
+__device__ __forceinline__ LaneGeom lane_geom(const JobGeom& jg, uint32_t g) {
+  LaneGeom lg;
+  const uint32_t tid = threadIdx.x;
+  lg.blk = tid >> 2;
+  lg.t = tid & 3u;
+  uint32_t gblk = g * kGroupBlocks + lg.blk;
+  lg.m_blk = gblk < jg.nb ? (gblk == jg.nb - 1 ? jg.m_last : (uint32_t)kL) : 0u;
+  int nv = (int)lg.m_blk - (int)(kSliceVals * lg.t);
+  lg.nv = (uint32_t)(nv < 0 ? 0 : (nv > kSliceVals ? kSliceVals : nv));
+  uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
+  lg.nfull = (uint32_t)((rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues) / kSliceVals);
+  lg.first = (uint64_t)gblk * kL + (uint64_t)kSliceVals * lg.t;
+  return lg;
+}
 
 // ---------------------------------------------------------------------------------------------------
 // shared memory
 // ---------------------------------------------------------------------------------------------------
-struct EncSmem {
-  uint32_t img[kImgWords];   // payload image of the outgoing group (zeroed, filled by OR)
-  uint32_t blk_mu[kGroupBlocks];
-  uint32_t blk_R[kGroupBlocks];     // 0 = constant or absent block
-  uint32_t blk_size[kGroupBlocks];  // record bytes, 0 = absent block
-  uint32_t prefix;                  // exclusive prefix of this group, in words
+// Dynamic shared memory of a CTA: this control block, then one or two `rows` buffers of kRowsBytes (one
+// padded 144-byte slice per thread: fp32 in, staged bytes, fp32 out).
+struct Smem {
+  alignas(128) uint32_t img[kImgWords];  // payload image of the incoming / outgoing group
+  uint32_t blk_size[kGroupBlocks];       // record bytes, 0 = absent block
+  uint32_t blk_R[kGroupBlocks];          // 0 = constant or absent block
+  uint32_t prefix;                       // exclusive prefix of this group, in words
   uint32_t fail;
 };
-struct DecSmem {
-  uint32_t img[kImgWords];  // payload image of the incoming group
-};
+constexpr int kCtlBytes = (sizeof(Smem) + 127) / 128 * 128;
+extern __shared__ __align__(128) uint8_t dyn_smem[];
+
+__device__ __forceinline__ void zero_image(uint32_t* img) {  // a barrier must follow
+  uint4* p = reinterpret_cast<uint4*>(img) + threadIdx.x;
+  constexpr int kVecs = kImgWords / 4, kFullRounds = kVecs / kThreads;
+#pragma unroll
+  for (int r = 0; r < kFullRounds; ++r) p[r * kThreads] = make_uint4(0u, 0u, 0u, 0u);
+  if (kFullRounds * kThreads + (int)threadIdx.x < kVecs) p[kFullRounds * kThreads] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
+// (128-bit streaming loads) and scatters them into the padded slices; in round r thread tid moves the
+// float4 number r*128 + tid of the group.  A __syncthreads must follow before the slices are read.
+__device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
+  const uint32_t cnt = (uint32_t)(rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues);
+  const float* src = x + (uint64_t)g * kGroupValues;
+  float4 t[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    if (4u * f + 4u <= cnt) {
+      t[r] = __ldcs(reinterpret_cast<const float4*>(src) + f);
+    } else {
+      t[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (4u * f + 0u < cnt) t[r].x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) t[r].y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) t[r].z = __ldcs(src + 4u * f + 2u);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    *reinterpret_cast<float4*>(rows + (f >> 3) * kSliceBytes + 16u * (f & 7u)) = t[r];
+  }
+}
+// Put the lane's 32 values (held in v) into its slice of the rows.
+__device__ __forceinline__ void write_slice(uint8_t* rows, const float4 (&v)[8]) {
+  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) slice[j] = v[j];
+}
+// Send the group's values from the rows to global memory with coalesced 128-bit streaming stores (the
+// mirror image of load_rows).  A __syncthreads must separate it from the writes of the slices.
+__device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
+  const uint32_t cnt = (uint32_t)(rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues);
+  float* dst = out + (uint64_t)g * kGroupValues;
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    const float4 t = *reinterpret_cast<const float4*>(rows + (f >> 3) * kSliceBytes + 16u * (f & 7u));
+    if (4u * f + 4u <= cnt) {
+      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+    } else {
+      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
+      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
+      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+    }
+  }
+}
 
 // ---------------------------------------------------------------------------------------------------
-// encode side: one block (rules R1-R8), values of the lane in x0..x3
+// encode side
 // ---------------------------------------------------------------------------------------------------
-// Outputs: R (0 = constant), mu_bits, the lane's stored bytes as a little-endian 16-byte string W[0..3]
-// (T bytes of it are meaningful), and the lane's lead-code byte.
+// Rules R1-R6 for the lane's block (the four lanes of a block compute the same plan).
+struct Plan {
+  uint32_t R;        // kept bits; 0 = constant (or absent) block, 32 = lossless
+  uint32_t mu_bits;  // representative value
+  float mu;
+  uint32_t sh;       // 32 - R (0 when R is 0 or 32)
+  uint32_t B;        // bytes per code
+  bool lossless;
+};
+
 template <bool kTail>
-__device__ __forceinline__ void encode_block(float x0, float x1, float x2, float x3, uint32_t m, uint32_t lane,
-                                             float eb, int eb_exp, uint32_t& mu_bits, uint32_t& R, uint32_t& W0,
-                                             uint32_t& W1, uint32_t& W2, uint32_t& W3, uint32_t& T,
-                                             uint32_t& code) {
-  int nv = 4;
+__device__ __forceinline__ Plan plan_block(float4 (&v)[8], const LaneGeom& lg, uint32_t lane, float eb, int eb_exp) {
   if (kTail) {
-    nv = (int)m - 4 * (int)lane;
-    nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
-    float f = __shfl_sync(kFull, x0, 0);  // element 0 always exists; it cannot change min or max
-    if (nv < 1) x0 = f;
-    if (nv < 2) x1 = f;
-    if (nv < 3) x2 = f;
-    if (nv < 4) x3 = f;
+    // values past the end of the data are replaced by the block's first value: they cannot change min or max
+    float f = __shfl_sync(kFull, v[0].x, lane & ~3u);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if ((uint32_t)(4 * j + 0) >= lg.nv) v[j].x = f;
+      if ((uint32_t)(4 * j + 1) >= lg.nv) v[j].y = f;
+      if ((uint32_t)(4 * j + 2) >= lg.nv) v[j].z = f;
+      if ((uint32_t)(4 * j + 3) >= lg.nv) v[j].w = f;
+    }
   }
+  float mx = max3_nan(max_nan(v[0].x, v[0].y), v[0].z, v[0].w);
+  float mn = min3_nan(min_nan(v[0].x, v[0].y), v[0].z, v[0].w);
+#pragma unroll
+  for (int j = 1; j < 8; ++j) {
+    mx = max3_nan(max3_nan(mx, v[j].x, v[j].y), v[j].z, v[j].w);
+    mn = min3_nan(min3_nan(mn, v[j].x, v[j].y), v[j].z, v[j].w);
+  }
+  mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 1));
+  mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 1));
+  mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 2));
+  mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 2));
   const float kInf = __uint_as_float(0x7f800000u);
-  float mx = warp_max_nan(max_nan(max_nan(x0, x1), max_nan(x2, x3)));
-  float mn = warp_min_nan(min_nan(min_nan(x0, x1), min_nan(x2, x3)));
   bool special = !(fabsf(mx) < kInf) || !(fabsf(mn) < kInf);  // NaN or Inf somewhere in the block
   float mu = __fadd_rn(__fmul_rn(0.5f, mn), __fmul_rn(0.5f, mx));
   uint32_t mub = __float_as_uint(mu);
   if ((mub << 1) == 0u) mub = 0u;  // a zero of either sign becomes +0
   mu = __uint_as_float(mub);
   float r = fmaxf(__fsub_rn(mx, mu), __fsub_rn(mu, mn));
-  W0 = W1 = W2 = W3 = 0u;
-  T = 0u;
-  code = 0u;
-  if (!special && r <= eb) {
-    R = 0u;
-    mu_bits = mub;
-    return;
+  Plan p;
+  if (lg.m_blk == 0u || (!special && r <= eb)) {
+    p.R = 0u;
+    p.mu_bits = mub;
+    p.mu = mu;
+    p.sh = 0u;
+    p.B = 0u;
+    p.lossless = false;
+    return p;
   }
   int m_bits = (int)((__float_as_uint(r) >> 23) & 0xffu) - eb_exp + 1;
-  bool lossless = special || m_bits >= 23;
-  R = lossless ? 32u : (uint32_t)(9 + m_bits);
-  if (lossless) {
-    mub = 0u;
-    mu = 0.0f;
+  p.lossless = special || m_bits >= 23;
+  p.R = p.lossless ? 32u : (uint32_t)(9 + m_bits);
+  p.mu_bits = p.lossless ? 0u : mub;
+  p.mu = __uint_as_float(p.mu_bits);
+  p.sh = 32u - p.R;
+  p.B = (p.R + 7u) >> 3;
+  return p;
+}
+
+__device__ __forceinline__ uint32_t code_of(float x, const Plan& p) {
+  return __float_as_uint(p.lossless ? x : __fsub_rn(x, p.mu)) >> p.sh;
+}
+
+// Rules R7-R8 for one quad of values with codes q0..q3 (prev = code before q0).  sa_e = 32 - 8*(stored
+// bytes of value e) is taken straight from the leading-zero count of (code xor predecessor): a value
+// stores its significant bytes; `fix` forces at least one stored byte when the field is 4 bytes wide
+// (lead is capped at 3).  Appends the quad's bytes to the lane's staging words and returns the new state.
+struct Stage {
+  uint32_t* wp;     // next staging word
+  uint32_t pendb;   // bits (0, 8, 16, 24) waiting in carry
+  uint32_t carry;   // the partial word, zero above pendb
+  uint32_t Tb;      // bits staged so far
+};
+__device__ __forceinline__ void append_quad(Stage& st, uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3,
+                                            uint32_t sa0, uint32_t sa1, uint32_t sa2, uint32_t sa3) {
+  // the stored (low) bytes of each code, most significant first, as little-endian integers ...
+  const uint32_t e0 = __funnelshift_rc(__byte_perm(q0, 0u, 0x0123), 0u, sa0);
+  const uint32_t e1 = __funnelshift_rc(__byte_perm(q1, 0u, 0x0123), 0u, sa1);
+  const uint32_t e2 = __funnelshift_rc(__byte_perm(q2, 0u, 0x0123), 0u, sa2);
+  const uint32_t e3 = __funnelshift_rc(__byte_perm(q3, 0u, 0x0123), 0u, sa3);
+  // ... concatenated into one 16-byte little-endian string W0..W3
+  const uint32_t s0 = 32u - sa0, s2 = 32u - sa2;
+  const uint32_t lo01 = e0 | __funnelshift_lc(0u, e1, s0), hi01 = __funnelshift_lc(e1, 0u, s0);
+  const uint32_t lo23 = e2 | __funnelshift_lc(0u, e3, s2), hi23 = __funnelshift_lc(e3, 0u, s2);
+  const uint32_t s01 = 64u - sa0 - sa1;  // bits of the first pair, 0..64
+  const bool upper = s01 >= 32u;
+  const uint32_t a = upper ? s01 - 32u : s01;
+  const uint32_t t0 = __funnelshift_lc(0u, lo23, a), t1 = __funnelshift_lc(lo23, hi23, a),
+                 t2 = __funnelshift_lc(hi23, 0u, a);
+  const uint32_t W0 = upper ? lo01 : (lo01 | t0);
+  const uint32_t W1 = upper ? (hi01 | t0) : (hi01 | t1);
+  const uint32_t W2 = upper ? t1 : t2;
+  const uint32_t W3 = upper ? t2 : 0u;
+  // append behind the bits waiting in carry; words past the end are overwritten by the next quad
+  const uint32_t z = st.pendb;
+  const uint32_t V0 = (W0 << z) | st.carry;
+  const uint32_t V1 = __funnelshift_l(W0, W1, z);
+  const uint32_t V2 = __funnelshift_l(W1, W2, z);
+  const uint32_t V3 = __funnelshift_l(W2, W3, z);
+  const uint32_t V4 = __funnelshift_l(W3, 0u, z);
+  st.wp[0] = V0;
+  st.wp[1] = V1;
+  st.wp[2] = V2;
+  st.wp[3] = V3;
+  const uint32_t T4b = 128u - sa0 - sa1 - sa2 - sa3;
+  const uint32_t totb = z + T4b;  // 0..152
+  const uint32_t c01 = (totb & 32u) ? V1 : V0, c23 = (totb & 32u) ? V3 : V2;
+  st.carry = (totb & 128u) ? V4 : ((totb & 64u) ? c23 : c01);
+  st.wp += totb >> 5;
+  st.pendb = totb & 31u;
+  st.Tb += T4b;
+}
+__device__ __forceinline__ void finish_stage(Stage& st) {
+  st.wp[0] = st.carry;  // the last partial word, zero padded
+  st.wp[1] = 0u;        // and a zero word behind it for the realigning copy
+}
+
+// Fast path: all 32 values valid, block not lossless, values in registers.
+__device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const float4 (&v)[8], const Plan& p, uint32_t prev,
+                                               uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  const uint32_t fix = (p.B == 4u) ? 1u : 0u;
+  const uint32_t cadj = (4u - p.B) * 85u;
+  const float mu = p.mu;
+  const uint32_t sh = p.sh;
+  Stage st = {slice, 0u, 0u, 0u};
+  code_lo = code_hi = 0u;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t q0 = __float_as_uint(__fsub_rn(v[j].x, mu)) >> sh, q1 = __float_as_uint(__fsub_rn(v[j].y, mu)) >> sh,
+                   q2 = __float_as_uint(__fsub_rn(v[j].z, mu)) >> sh, q3 = __float_as_uint(__fsub_rn(v[j].w, mu)) >> sh;
+    const uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
+                   sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
+    prev = q3;
+    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field
+    const uint32_t cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) >> 3) - cadj;
+    if (j < 4)
+      code_lo |= cb << (8 * j);
+    else
+      code_hi |= cb << (8 * (j - 4));
+    append_quad(st, q0, q1, q2, q3, sa0, sa1, sa2, sa3);
   }
-  mu_bits = mub;
-  uint32_t sh = 32u - R;
-  uint32_t q0 = __float_as_uint(lossless ? x0 : __fsub_rn(x0, mu)) >> sh;
-  uint32_t q1 = __float_as_uint(lossless ? x1 : __fsub_rn(x1, mu)) >> sh;
-  uint32_t q2 = __float_as_uint(lossless ? x2 : __fsub_rn(x2, mu)) >> sh;
-  uint32_t q3 = __float_as_uint(lossless ? x3 : __fsub_rn(x3, mu)) >> sh;
-  uint32_t B = (R + 7u) >> 3;
-  uint32_t min_nb = (B == 4u) ? 1u : 0u;  // lead is capped at 3, so a 4-byte field always stores a byte
-  uint32_t p0 = __shfl_up_sync(kFull, q3, 1);
-  if (lane == 0) p0 = 0u;
-  // stored bytes of an element = significant bytes of (q xor predecessor)
-  uint32_t nb0 = max((39u - (uint32_t)__clz(q0 ^ p0)) >> 3, min_nb);
-  uint32_t nb1 = max((39u - (uint32_t)__clz(q1 ^ q0)) >> 3, min_nb);
-  uint32_t nb2 = max((39u - (uint32_t)__clz(q2 ^ q1)) >> 3, min_nb);
-  uint32_t nb3 = max((39u - (uint32_t)__clz(q3 ^ q2)) >> 3, min_nb);
-  if (kTail) {
-    uint32_t l0 = B - nb0, l1 = B - nb1, l2 = B - nb2, l3 = B - nb3;
-    if (nv < 1) nb0 = 0u, l0 = 0u;
-    if (nv < 2) nb1 = 0u, l1 = 0u;
-    if (nv < 3) nb2 = 0u, l2 = 0u;
-    if (nv < 4) nb3 = 0u, l3 = 0u;
-    code = l0 | (l1 << 2) | (l2 << 4) | (l3 << 6);
-  } else {
-    code = B * 0x55u - (nb0 + 4u * nb1 + 16u * nb2 + 64u * nb3);
+  finish_stage(st);
+  T_out = st.Tb >> 3;
+}
+
+// General path (ragged slices, lossless blocks): rolled loop over the quads, values re-read from the slice.
+// Staging in place is safe: quad j is read before anything is written at or behind its position.
+__device__ __noinline__ void emit_lane_slow(uint32_t* slice, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
+                                            uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  const bool lossless = R == 32u;
+  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
+  const uint32_t fix = (B == 4u) ? 1u : 0u;
+  const float mu = __uint_as_float(mu_bits);
+  Stage st = {slice, 0u, 0u, 0u};
+  uint64_t codes = 0ull;
+  const float4* src = reinterpret_cast<const float4*>(slice);
+#pragma unroll 1
+  for (uint32_t j = 0; j < 8u; ++j) {
+    const float4 x = src[j];
+    const uint32_t q0 = __float_as_uint(lossless ? x.x : __fsub_rn(x.x, mu)) >> sh,
+                   q1 = __float_as_uint(lossless ? x.y : __fsub_rn(x.y, mu)) >> sh,
+                   q2 = __float_as_uint(lossless ? x.z : __fsub_rn(x.z, mu)) >> sh,
+                   q3 = __float_as_uint(lossless ? x.w : __fsub_rn(x.w, mu)) >> sh;
+    uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
+             sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
+    prev = q3;
+    uint32_t l0 = (sa0 >> 3) - (4u - B), l1 = (sa1 >> 3) - (4u - B), l2 = (sa2 >> 3) - (4u - B), l3 = (sa3 >> 3) - (4u - B);
+    if (4u * j + 0u >= nv) sa0 = 32u, l0 = 0u;  // values past the end store nothing and have code 0
+    if (4u * j + 1u >= nv) sa1 = 32u, l1 = 0u;
+    if (4u * j + 2u >= nv) sa2 = 32u, l2 = 0u;
+    if (4u * j + 3u >= nv) sa3 = 32u, l3 = 0u;
+    codes |= (uint64_t)(l0 | (l1 << 2) | (l2 << 4) | (l3 << 6)) << (8u * j);
+    append_quad(st, q0, q1, q2, q3, sa0, sa1, sa2, sa3);
   }
-  T = nb0 + nb1 + nb2 + nb3;
-  // the low nb bytes of q, most significant first, as a little-endian integer
-  uint32_t e0 = __funnelshift_rc(__byte_perm(q0, 0u, 0x0123), 0u, 32u - 8u * nb0);
-  uint32_t e1 = __funnelshift_rc(__byte_perm(q1, 0u, 0x0123), 0u, 32u - 8u * nb1);
-  uint32_t e2 = __funnelshift_rc(__byte_perm(q2, 0u, 0x0123), 0u, 32u - 8u * nb2);
-  uint32_t e3 = __funnelshift_rc(__byte_perm(q3, 0u, 0x0123), 0u, 32u - 8u * nb3);
-  uint32_t s0 = 8u * nb0, s2 = 8u * nb2;
-  uint32_t lo01 = e0 | __funnelshift_lc(0u, e1, s0), hi01 = __funnelshift_lc(e1, 0u, s0);
-  uint32_t lo23 = e2 | __funnelshift_lc(0u, e3, s2), hi23 = __funnelshift_lc(e3, 0u, s2);
-  uint32_t s = 8u * (nb0 + nb1);
-  bool upper = s >= 32u;
-  uint32_t a = upper ? s - 32u : s;
-  uint32_t t0 = __funnelshift_lc(0u, lo23, a), t1 = __funnelshift_lc(lo23, hi23, a),
-           t2 = __funnelshift_lc(hi23, 0u, a);
-  W0 = upper ? lo01 : (lo01 | t0);
-  W1 = upper ? (hi01 | t0) : (hi01 | t1);
-  W2 = upper ? t1 : t2;
-  W3 = upper ? t2 : 0u;
+  finish_stage(st);
+  T_out = st.Tb >> 3;
+  code_lo = (uint32_t)codes;
+  code_hi = (uint32_t)(codes >> 32);
 }
 
-// The image is zeroed once and then filled ONLY by atomic OR, so bytes of one word may come from any lane.
-__device__ __forceinline__ void or_byte(uint32_t* img, uint32_t off, uint32_t byte) {
-  atomicOr(&img[off >> 2], (byte & 0xffu) << (8u * (off & 3u)));
+// Copy the lane's T staged bytes from its slice to byte offset dst of the image.  The first and last image
+// word may be shared with a neighbour and are ORed in; the words between are plain stores.
+__device__ __forceinline__ void copy_staged(uint32_t* img, const uint32_t* slice, uint32_t dst, uint32_t T) {
+  if (T == 0u) return;
+  const uint32_t z = 8u * (dst & 3u);
+  uint32_t* out = img + (dst >> 2);
+  const uint32_t nw = ((dst & 3u) + T + 3u) >> 2;  // image words touched
+  atomicOr(&out[0], slice[0] << z);
+  if (nw > 1u) atomicOr(&out[nw - 1u], __funnelshift_l(slice[nw - 2u], slice[nw - 1u], z));
+  if (nw <= 2u) return;
+  const uint32_t ni = nw - 2u;  // interior words 1 .. nw-2
+  const uint4* src = reinterpret_cast<const uint4*>(slice);
+  uint32_t prevw = 0u;
+  for (uint32_t c = 0; 4u * c <= ni; ++c) {
+    const uint4 cur = src[c];
+    const uint32_t w0 = __funnelshift_l(prevw, cur.x, z), w1 = __funnelshift_l(cur.x, cur.y, z),
+                   w2 = __funnelshift_l(cur.y, cur.z, z), w3 = __funnelshift_l(cur.z, cur.w, z);
+    prevw = cur.w;
+    const uint32_t g = 4u * c;  // image word of w0; word g is interior iff g - 1 < ni (unsigned)
+    if (g - 1u < ni) out[g] = w0;
+    if (g < ni) out[g + 1u] = w1;
+    if (g + 1u < ni) out[g + 2u] = w2;
+    if (g + 2u < ni) out[g + 3u] = w3;
+  }
 }
 
-// OR a lane's T-byte string into the image at byte offset off.
-__device__ __forceinline__ void place_string(uint32_t* img, uint32_t off, uint32_t T, uint32_t W0, uint32_t W1,
-                                             uint32_t W2, uint32_t W3) {
-  uint32_t z = 8u * (off & 3u);
-  uint32_t wi = off >> 2;
-  uint32_t cnt = ((off & 3u) + T + 3u) >> 2;
-  uint32_t V0 = W0 << z;
-  uint32_t V1 = __funnelshift_l(W0, W1, z);
-  uint32_t V2 = __funnelshift_l(W1, W2, z);
-  uint32_t V3 = __funnelshift_l(W2, W3, z);
-  uint32_t V4 = __funnelshift_l(W3, 0u, z);
-  if (cnt > 0) atomicOr(&img[wi], V0);
-  if (cnt > 1) atomicOr(&img[wi + 1], V1);
-  if (cnt > 2) atomicOr(&img[wi + 2], V2);
-  if (cnt > 3) atomicOr(&img[wi + 3], V3);
-  if (cnt > 4) atomicOr(&img[wi + 4], V4);
-}
-
-// inclusive warp scan of three 10-bit fields packed in one word
-__device__ __forceinline__ uint32_t warp_scan_packed(uint32_t v, uint32_t lane) {
+// inclusive warp scan
+__device__ __forceinline__ uint32_t warp_scan_u32(uint32_t v, uint32_t lane) {
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
     uint32_t t = __shfl_up_sync(kFull, v, d);
@@ -211,159 +430,135 @@ __device__ __forceinline__ uint32_t warp_scan_packed(uint32_t v, uint32_t lane) 
   }
   return v;
 }
-__device__ __forceinline__ uint32_t warp_scan_u32(uint32_t v, uint32_t lane) { return warp_scan_packed(v, lane); }
-
-// Decoupled look-back over the groups of one job (tile order = blockIdx.x order, which is the order CTAs
-// are issued in).  Called by all lanes of warp 0.  Returns false if it gave up; every wait is bounded.
-__device__ __forceinline__ bool lookback(uint64_t* state, uint32_t g, uint32_t words, uint32_t epoch,
-                                         uint32_t lane, uint32_t* status, uint32_t& excl_out) {
-  if (g == 0) {
-    if (lane == 0) st_relaxed_u64(&state[0], pack_state(epoch, kFlagPrefix, words));
-    excl_out = 0;
-    return true;
-  }
-  if (lane == 0) st_relaxed_u64(&state[g], pack_state(epoch, kFlagAggregate, words));
-  uint32_t excl = 0;
-  int base = (int)g - 1;
-  uint32_t spins = 0;
-  bool ok = true;
-  while (true) {
-    int t = base - (int)lane;
-    uint32_t flag = kFlagPrefix, value = 0;  // tiles before the first one: an empty prefix
-    if (t >= 0) {
-      uint64_t w = ld_relaxed_u64(&state[t]);
-      flag = ((uint32_t)(w >> 32) == epoch) ? (uint32_t)(w >> 30) & 3u : 0u;
-      value = (uint32_t)w & kValueMask;
-    }
-    uint32_t ready = __ballot_sync(kFull, flag != 0u);
-    uint32_t closed = __ballot_sync(kFull, flag == kFlagPrefix || flag == kFlagPoison);
-    uint32_t first = closed ? (uint32_t)__ffs(closed) - 1u : 32u;
-    uint32_t need = (first >= 31u) ? kFull : ((2u << first) - 1u);
-    if ((ready & need) == need) {
-      uint32_t poison = __ballot_sync(kFull, flag == kFlagPoison) & need;
-      uint32_t v = ((need >> lane) & 1u) ? value : 0u;
-      excl += __reduce_add_sync(kFull, v);
-      if (poison) {
-        ok = false;
-        break;
-      }
-      if (first != 32u) break;
-      base -= 32;
-      continue;
-    }
-    if (++spins > kSpinLimit) {
-      ok = false;
-      if (lane == 0) raise(status, kErrTimeout);
-      break;
-    }
-    __nanosleep(64);
-  }
-  if (lane == 0)
-    st_relaxed_u64(&state[g], ok ? pack_state(epoch, kFlagPrefix, excl + words) : pack_state(epoch, kFlagPoison, 0));
-  excl_out = excl;
-  return ok;
+// inclusive scan over the four lanes of a block; total = sum over the quad
+__device__ __forceinline__ uint32_t quad_scan(uint32_t v, uint32_t t, uint32_t lane, uint32_t& total) {
+  uint32_t a = __shfl_up_sync(kFull, v, 1);
+  if (t >= 1u) v += a;
+  a = __shfl_up_sync(kFull, v, 2);
+  if (t >= 2u) v += a;
+  total = __shfl_sync(kFull, v, lane | 3u);
+  return v;
 }
 
-// Encode the 8 blocks a warp holds in v[], build the group image, find the group's place in the stream
-// and copy it out.  cnt = blocks this warp owns in the group; nblk = blocks in the group.
-__device__ __forceinline__ void encode_group(EncSmem& sm, float4 (&v)[kWarpBlocks], const EncodeBatch& b,
-                                             const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout) {
+// Place of a group in its stream = sum of the sizes of all groups before it.  A chained look-back (wait
+// for the predecessor's inclusive prefix) advances at most one window of tiles per L2 round trip, which
+// caps a kernel of 8192 tiles at ~100 us whatever its work.  Instead sizes are summed on two levels and
+// nothing ever waits on a prefix: A[t] = size of tile t; SA[s] = size of super-tile s (32 tiles), written
+// by the super-tile's last tile from the A's it has to read anyway.  Tile g needs A[32s .. g-1] and
+// SA[0 .. s-1]: independent loads spread over the CTA's threads, one round trip once the data is there.
+// Words carry the launch's epoch, so stale entries read as "not written yet"; every wait is bounded.
+__device__ __forceinline__ uint32_t poll_size(const uint64_t* p, uint32_t epoch, uint32_t* status, bool& bad) {
+  uint32_t spins = 0;
+  while (true) {
+    const uint64_t w = ld_relaxed_u64(p);
+    if ((uint32_t)(w >> 32) == epoch) {
+      if (((uint32_t)(w >> 30) & 3u) == kFlagPoison) bad = true;
+      return (uint32_t)w & kValueMask;
+    }
+    if (++spins > kSpinLimit) {
+      raise(status, kErrTimeout);
+      bad = true;
+      return 0u;
+    }
+    __nanosleep(32);
+  }
+}
+// Called by every thread of the CTA after A[g] was published.  Adds the group's exclusive prefix (in words)
+// to sm.prefix and raises sm.fail on a poisoned or timed-out entry; both are read after the next barrier.
+__device__ __forceinline__ void find_prefix(Smem& sm, uint64_t* A, uint64_t* SA, uint32_t g, uint32_t G, uint32_t words,
+                                            uint32_t epoch, uint32_t* status) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  const uint32_t nblk = min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks);
-  const int cnt = max(0, min(kWarpBlocks, (int)nblk - (int)(warp * kWarpBlocks)));
-  const uint32_t last_blk = jg.nb - 1 - g * kGroupBlocks;  // group-relative index of the job's last block
+  const uint32_t s = g >> 5, r = g & 31u;
+  uint32_t sum = 0u;
+  bool bad = false;
+  if (warp == 0) {
+    if (lane < r) sum = poll_size(&A[32u * s + lane], epoch, status, bad);
+    sum = __reduce_add_sync(kFull, sum);
+    bad = __any_sync(kFull, bad);
+    if (lane == 0) {
+      if (r == 31u || g == G - 1u)
+        st_relaxed_u64(&SA[s], pack_state(epoch, bad ? kFlagPoison : kFlagAggregate, sum + words));
+      if (sum) atomicAdd(&sm.prefix, sum);
+      if (bad) atomicOr(&sm.fail, 1u);
+    }
+  } else {
+    for (uint32_t t = tid - 32u; t < s; t += kThreads - 32u) sum += poll_size(&SA[t], epoch, status, bad);
+    sum = __reduce_add_sync(kFull, sum);
+    bad = __any_sync(kFull, bad);
+    if (lane == 0) {
+      if (sum) atomicAdd(&sm.prefix, sum);
+      if (bad) atomicOr(&sm.fail, 1u);
+    }
+  }
+}
 
-  uint32_t W[kWarpBlocks][4];
-  uint32_t tp[3] = {0u, 0u, 0u};  // per-lane stored-byte counts of the 8 blocks, three 10-bit fields per word
-  uint32_t codes[2] = {0u, 0u};   // per-lane lead-code bytes of the 8 blocks
-  uint32_t R_mine = 0u, mu_mine = 0u;  // lane i keeps R and mu of the warp's block i
-#pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    W[i][0] = W[i][1] = W[i][2] = W[i][3] = 0u;
-    if (i < cnt) {
-      uint32_t blk = warp * kWarpBlocks + i;
-      uint32_t mu_bits, R, T, code;
-      if (blk == last_blk && jg.m_last != (uint32_t)kL)
-        encode_block<true>(v[i].x, v[i].y, v[i].z, v[i].w, jg.m_last, lane, b.eb, b.eb_exp, mu_bits, R, W[i][0],
-                           W[i][1], W[i][2], W[i][3], T, code);
-      else
-        encode_block<false>(v[i].x, v[i].y, v[i].z, v[i].w, kL, lane, b.eb, b.eb_exp, mu_bits, R, W[i][0], W[i][1],
-                            W[i][2], W[i][3], T, code);
-      tp[i / 3] |= T << (10 * (i % 3));
-      codes[i / 4] |= code << (8 * (i % 4));
-      if (lane == (uint32_t)i) {
-        R_mine = R;
-        mu_mine = mu_bits;
-      }
-    }
+// Encode the group whose values the threads hold in v[] (32 per thread), build its payload image, find its
+// place in the stream and copy it out.  The image must have been zeroed (and that made visible by the
+// barrier inside) before the call.
+__device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v)[8], const LaneGeom& lg,
+                                             const EncodeBatch& b, const JobGeom& jg, uint32_t g, uint32_t y,
+                                             uint8_t* sout) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  uint32_t* slice = reinterpret_cast<uint32_t*>(rows + tid * kSliceBytes);
+  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
+
+  Plan p = tail ? plan_block<true>(v, lg, lane, b.eb, b.eb_exp) : plan_block<false>(v, lg, lane, b.eb, b.eb_exp);
+  // code of the value just before this lane's first one (0 at the start of a block)
+  uint32_t prev = __shfl_up_sync(kFull, code_of(v[7].w, p), 1);
+  if (lg.t == 0u) prev = 0u;
+  uint32_t T = 0u, code_lo = 0u, code_hi = 0u;
+  if (p.R != 0u) {
+    if (tail || p.lossless)
+      emit_lane_slow(slice, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
+    else
+      emit_lane_fast(slice, v, p, prev, T, code_lo, code_hi);
   }
-  // exclusive offsets of every lane's bytes inside its block's record, and the records' sizes
-  uint32_t incl[3], tot[3];
-#pragma unroll
-  for (int k = 0; k < 3; ++k) {
-    incl[k] = warp_scan_packed(tp[k], lane);
-    tot[k] = __shfl_sync(kFull, incl[k], 31);
+  uint32_t total;
+  const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
+  const uint32_t cbytes = (lg.m_blk + 3u) >> 2;  // lead-code bytes of the block
+  if (lg.t == 0u) {
+    sm.blk_size[lg.blk] = lg.m_blk == 0u ? 0u : (p.R ? 5u + cbytes + total : 4u);
+    sm.blk_R[lg.blk] = p.R;
   }
-  if (lane < (uint32_t)kWarpBlocks) {
-    uint32_t blk = warp * kWarpBlocks + lane;
-    uint32_t size = 0u;
-    if ((int)lane < cnt) {
-      uint32_t total = (tot[lane / 3] >> (10 * (lane % 3))) & 0x3ffu;
-      uint32_t m = (blk == last_blk) ? jg.m_last : (uint32_t)kL;
-      size = R_mine ? 5u + ((m + 3u) >> 2) + total : 4u;
-    }
-    sm.blk_mu[blk] = mu_mine;
-    sm.blk_R[blk] = R_mine;
-    sm.blk_size[blk] = size;
-  }
-  __syncthreads();  // also orders the zero-fill of the image before the ORs below
+  __syncthreads();  // sizes visible; also: image zero-fill and all staging done
 
   // every warp derives the offsets of all 32 records (cheap, and saves a barrier)
-  uint32_t my_size = sm.blk_size[lane];
-  uint32_t my_R = sm.blk_R[lane];
-  uint32_t bitmap = __ballot_sync(kFull, my_R != 0u);
-  uint32_t k = (uint32_t)__popc(bitmap);
-  uint32_t incl_sz = warp_scan_u32(my_size, lane);
-  uint32_t my_off = 2u * k + incl_sz - my_size;
-  uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
-  uint32_t words = (raw + 3u) >> 2;
+  const uint32_t sz_l = sm.blk_size[lane];
+  const uint32_t R_l = sm.blk_R[lane];
+  const uint32_t bitmap = __ballot_sync(kFull, R_l != 0u);
+  const uint32_t k = (uint32_t)__popc(bitmap);
+  const uint32_t incl_sz = warp_scan_u32(sz_l, lane);
+  const uint32_t off_l = 2u * k + incl_sz - sz_l;
+  const uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
+  const uint32_t words = (raw + 3u) >> 2;
+  const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
 
+  uint64_t* A = b.tile_state + (uint64_t)y * b.state_stride;
+  uint64_t* SA = A + b.tiles_per_job;
   if (warp == 0) {
-    if (my_R != 0u) {
+    if (lane == 0) st_relaxed_u64(&A[g], pack_state(b.epoch, kFlagAggregate, words));
+    if (R_l != 0u) {
       uint32_t rank = (uint32_t)__popc(bitmap & ((1u << lane) - 1u));
-      atomicOr(&sm.img[rank >> 1], my_size << (16u * (rank & 1u)));
+      atomicOr(&sm.img[rank >> 1], sz_l << (16u * (rank & 1u)));
     }
   }
-#pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    if (i < cnt) {
-      uint32_t blk = warp * kWarpBlocks + i;
-      uint32_t off = __shfl_sync(kFull, my_off, blk);
-      uint32_t R = sm.blk_R[blk];
-      uint32_t mu_bits = sm.blk_mu[blk];
-      if (R == 0u) {
-        if (lane < 4u) or_byte(sm.img, off + lane, mu_bits >> (8u * lane));
-      } else {
-        uint32_t m = (blk == last_blk) ? jg.m_last : (uint32_t)kL;
-        uint32_t cb = (m + 3u) >> 2;
-        if (lane < 5u) or_byte(sm.img, off + lane, (lane < 4u) ? (mu_bits >> (8u * lane)) : R);
-        if (lane < cb) or_byte(sm.img, off + 5u + lane, codes[i / 4] >> (8 * (i % 4)));
-        uint32_t T = (tp[i / 3] >> (10 * (i % 3))) & 0x3ffu;
-        uint32_t excl = ((incl[i / 3] >> (10 * (i % 3))) & 0x3ffu) - T;
-        place_string(sm.img, off + 5u + cb + excl, T, W[i][0], W[i][1], W[i][2], W[i][3]);
-      }
+  if (lg.m_blk != 0u) {
+    if (lg.t == 0u) {
+      or_u32(sm.img, boff, p.mu_bits);
+      if (p.R) or_u8(sm.img, boff + 4u, p.R);
+    }
+    if (p.R) {
+      if (8u * lg.t < cbytes) or_u64(sm.img, boff + 5u + 8u * lg.t, code_lo, code_hi);
+      copy_staged(sm.img, slice, boff + 5u + cbytes + excl, T);
     }
   }
 
   // place of the group in the stream
-  if (warp == 0) {
-    uint32_t excl;
-    bool ok = lookback(b.tile_state + (uint64_t)y * b.tiles_per_job, g, words, b.epoch, lane, b.status, excl);
-    if (lane == 0) {
-      sm.prefix = excl;
-      sm.fail = ok ? 0u : 1u;
-    }
-  }
+#ifdef CCOLL_EXP_NOPREFIX
+  if (threadIdx.x == 0) sm.prefix = g * words;
+#else
+  find_prefix(sm, A, SA, g, jg.G, words, b.epoch, b.status);
+#endif
   __syncthreads();
   const uint32_t prefix = sm.prefix;
   if (sm.fail) return;
@@ -374,11 +569,22 @@ __device__ __forceinline__ void encode_group(EncSmem& sm, float4 (&v)[kWarpBlock
     if (tid == 0) raise(b.status, kErrCapacity);
     return;
   }
-  uint32_t* dst = out32 + (base >> 2) + prefix;
-  for (uint32_t j = tid; j < words; j += kThreads) dst[j] = sm.img[j];
+  {
+    // coalesced copy-out: single words up to the first 16-byte boundary of the stream, then 128-bit stores
+    uint32_t* dst = out32 + (base >> 2) + prefix;
+    const uint32_t head = min(words, (4u - (((base >> 2) + prefix) & 3u)) & 3u);
+    if (tid < head) dst[tid] = sm.img[tid];
+    const uint32_t nvec = (words - head) >> 2;
+    uint4* dst4 = reinterpret_cast<uint4*>(dst + head);
+    const uint32_t* src = sm.img + head;
+    for (uint32_t i = tid; i < nvec; i += kThreads)
+      dst4[i] = make_uint4(src[4u * i], src[4u * i + 1u], src[4u * i + 2u], src[4u * i + 3u]);
+    const uint32_t done = head + 4u * nvec;
+    if (tid < words - done) dst[done + tid] = sm.img[done + tid];
+  }
   if (tid == 0) {
-    out32[8 + g] = prefix;                 // dir[g]
-    out32[8 + jg.G + 1 + g] = bitmap;      // bitmap[g]
+    out32[8 + g] = prefix;             // dir[g]
+    out32[8 + jg.G + 1 + g] = bitmap;  // bitmap[g]
   }
   if (g == 0 && tid >= 32 && tid < 32 + 4) {
     // static part of the header and the zero pad between the bitmap and the payload
@@ -424,32 +630,6 @@ __device__ __forceinline__ void write_empty_stream(const EncodeBatch& b, uint32_
   if (b.moved) atomicAdd(reinterpret_cast<unsigned long long*>(b.moved), (unsigned long long)b.moved_mult * 48ull);
 }
 
-__device__ __forceinline__ void zero_image(uint32_t* img) {
-  uint4* p = reinterpret_cast<uint4*>(img);
-  for (uint32_t j = threadIdx.x; j < (uint32_t)kImgWords / 4; j += kThreads) p[j] = make_uint4(0u, 0u, 0u, 0u);
-}
-
-// Load the (up to) 8 blocks a warp owns: one 128-bit streaming load per lane and block.
-__device__ __forceinline__ void load_blocks(const float* x, const JobGeom& jg, uint32_t g, float4 (&v)[kWarpBlocks]) {
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    uint32_t gblk = g * kGroupBlocks + warp * kWarpBlocks + i;
-    v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (gblk < jg.nb) {
-      const float* p = x + (uint64_t)gblk * kL + 4u * lane;
-      uint32_t m = (gblk == jg.nb - 1) ? jg.m_last : (uint32_t)kL;
-      if (4u * lane + 4u <= m) {
-        v[i] = __ldcs(reinterpret_cast<const float4*>(p));
-      } else {
-        if (4u * lane + 0u < m) v[i].x = __ldcs(p + 0);
-        if (4u * lane + 1u < m) v[i].y = __ldcs(p + 1);
-        if (4u * lane + 2u < m) v[i].z = __ldcs(p + 2);
-      }
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------------------
 // decode side
 // ---------------------------------------------------------------------------------------------------
@@ -484,200 +664,213 @@ __device__ __forceinline__ bool open_group(const uint8_t* sin, uint64_t in_bytes
   return true;
 }
 
-// Decode the blocks this warp owns in group g into v[].  Returns false (for the whole CTA) on a corrupt group.
-__device__ __forceinline__ bool decode_group(DecSmem& sm, const StreamView& sv, const JobGeom& jg, uint32_t g,
-                                             float4 (&v)[kWarpBlocks]) {
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  const uint32_t nblk = min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks);
-  const int cnt = max(0, min(kWarpBlocks, (int)nblk - (int)(warp * kWarpBlocks)));
-  const uint32_t last_blk = jg.nb - 1 - g * kGroupBlocks;
+// sum of the 2-bit fields of a 64-bit word
+__device__ __forceinline__ uint32_t sum_fields2(uint32_t lo, uint32_t hi) {
+  return (uint32_t)(__popc(lo & 0x55555555u) + __popc(hi & 0x55555555u)) +
+         2u * (uint32_t)(__popc(lo & 0xaaaaaaaau) + __popc(hi & 0xaaaaaaaau));
+}
 
-  // stage the group's payload in shared memory
-  const uint32_t* src = sv.words + (sv.base >> 2) + sv.a;
-  for (uint32_t j = tid; j < sv.gw; j += kThreads) sm.img[j] = __ldcs(src + j);
-  __syncthreads();
+// Decode the lane's 32 values of group g into v[].  Returns false (for the whole CTA) on a corrupt group.
+// The group's payload must already be staged in sm.img (and visible).  nblk = blocks in the group.
+__device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
+                                             float4 (&v)[8]) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  const uint32_t* img = sm.img;
+  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
 
   // offsets of the 32 records: lane b looks at block b
   bool bad = false;
   const uint32_t map = sv.map;
   const uint32_t k = (uint32_t)__popc(map);
-  uint32_t my_size = 0u;
+  uint32_t sz_l = 0u;
   if (lane < nblk) {
     if ((map >> lane) & 1u) {
       uint32_t rank = (uint32_t)__popc(map & ((1u << lane) - 1u));
-      my_size = (rank < 2u * sv.gw) ? reinterpret_cast<const uint16_t*>(sm.img)[rank] : 0u;
+      sz_l = (rank < 2u * sv.gw) ? reinterpret_cast<const uint16_t*>(img)[rank] : 0u;
     } else {
-      my_size = 4u;
+      sz_l = 4u;
     }
   }
-  uint32_t incl_sz = warp_scan_u32(my_size, lane);
-  uint32_t my_off = 2u * k + incl_sz - my_size;
-  uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
-  if (((raw + 3u) >> 2) != sv.gw) bad = true;
+  const uint32_t incl_sz = warp_scan_u32(sz_l, lane);
+  const uint32_t off_l = 2u * k + incl_sz - sz_l;
+  const uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
+  if (((raw + 3u) >> 2) != sv.gw) bad = true;  // the same verdict in every thread
+  const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
+  const uint32_t size_blk = __shfl_sync(kFull, sz_l, lg.blk);
+  const bool nonconst = lg.m_blk != 0u && ((map >> lg.blk) & 1u);
 
-  // headers and lead codes of this warp's blocks, then one packed scan for all of them
-  uint32_t tp[3] = {0u, 0u, 0u};
-  uint32_t codes[2] = {0u, 0u};
-  if (!bad) {
-#pragma unroll
-    for (int i = 0; i < kWarpBlocks; ++i) {
-      if (i < cnt) {
-        uint32_t blk = warp * kWarpBlocks + i;
-        if ((map >> blk) & 1u) {
-          uint32_t off = __shfl_sync(kFull, my_off, blk);
-          uint32_t R = img_u8(sm.img, off + 4u);
-          uint32_t B = (R + 7u) >> 3;
-          if (!((R >= 10u && R <= 32u))) bad = true;
-          uint32_t m = (blk == last_blk) ? jg.m_last : (uint32_t)kL;
-          uint32_t cb = (m + 3u) >> 2;
-          uint32_t code = (lane < cb && !bad) ? img_u8(sm.img, off + 5u + lane) : 0u;
-          int nv = (int)m - 4 * (int)lane;
-          nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
-          uint32_t T = 0u;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t lead = (code >> (2 * j)) & 3u;
-            if (j < nv) {
-              if (lead > B) bad = true;
-              T += B - lead;
-            } else if (lead) {
-              bad = true;
-            }
+  // header, lead codes and stored-byte count of the lane
+  uint32_t R = 0u, B = 0u, code_lo = 0u, code_hi = 0u, T = 0u;
+  const uint32_t cbytes = (lg.m_blk + 3u) >> 2;
+  if (!bad && nonconst) {
+    R = img_u8(img, boff + 4u);
+    if (!(R >= 10u && R <= 32u)) bad = true;
+    B = (R + 7u) >> 3;
+    if (8u * lg.t < cbytes) {
+      uint32_t o = boff + 5u + 8u * lg.t;
+      uint32_t w = o >> 2, z = 8u * (o & 3u);
+      uint32_t a0 = img[w], a1 = img[w + 1], a2 = img[w + 2];
+      code_lo = __funnelshift_r(a0, a1, z);
+      code_hi = __funnelshift_r(a1, a2, z);
+      if (tail) {
+        // only cbytes code bytes exist; codes of values past the end must be zero
+        uint32_t vb = cbytes - 8u * lg.t;  // valid code bytes of this lane (>= 1)
+        if (vb < 8u) {
+          if (vb <= 4u) {
+            code_hi = 0u;
+            if (vb < 4u) code_lo &= (1u << (8u * vb)) - 1u;
+          } else {
+            code_hi &= (1u << (8u * (vb - 4u))) - 1u;
           }
-          if (bad) T = 0u;
-          tp[i / 3] |= (T & 0x3ffu) << (10 * (i % 3));
-          codes[i / 4] |= code << (8 * (i % 4));
+        }
+        if (lg.nv < (uint32_t)kSliceVals) {
+          uint64_t c = ((uint64_t)code_hi << 32) | code_lo;
+          if (c >> (2u * lg.nv)) bad = true;
         }
       }
     }
+    if (B == 2u && ((code_lo & (code_lo >> 1) & 0x55555555u) | (code_hi & (code_hi >> 1) & 0x55555555u)))
+      bad = true;  // lead 3 cannot occur in a 2-byte field
+    T = B * lg.nv - sum_fields2(code_lo, code_hi);
+    if (bad) T = 0u;
   }
-  bad = __any_sync(kFull, bad);
-  uint32_t incl[3], tot[3];
-#pragma unroll
-  for (int kk = 0; kk < 3; ++kk) {
-    incl[kk] = warp_scan_packed(tp[kk], lane);
-    tot[kk] = __shfl_sync(kFull, incl[kk], 31);
-  }
-  if (!bad) {
-#pragma unroll
-    for (int i = 0; i < kWarpBlocks; ++i) {
-      if (i < cnt) {
-        uint32_t blk = warp * kWarpBlocks + i;
-        if ((map >> blk) & 1u) {
-          uint32_t m = (blk == last_blk) ? jg.m_last : (uint32_t)kL;
-          uint32_t size = __shfl_sync(kFull, my_size, blk);
-          uint32_t total = (tot[i / 3] >> (10 * (i % 3))) & 0x3ffu;
-          if (size != 5u + ((m + 3u) >> 2) + total) bad = true;
-        }
-      }
-    }
-  }
+  uint32_t total;
+  const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
+  if (nonconst && !bad && size_blk != 5u + cbytes + total) bad = true;
   if (__syncthreads_or(bad ? 1 : 0)) return false;
 
+  // Summary of the lane's values for the predecessor chain: for each byte of the code field, the byte the
+  // LAST value of the lane that stores it holds (found from the lead codes alone, then fetched).
+  const uint32_t pos0 = boff + 5u + cbytes + excl;  // image offset of the lane's first stored byte
+  uint32_t sval = 0u, smask = 0u;
+  if (nonconst && lg.nv != 0u) {
+    const uint32_t f0lo = code_lo & 0x55555555u, f1lo = (code_lo >> 1) & 0x55555555u;
+    const uint32_t f0hi = code_hi & 0x55555555u, f1hi = (code_hi >> 1) & 0x55555555u;
+    uint32_t vlo = 0x55555555u, vhi = 0x55555555u;  // valid values of the lane, one bit per 2-bit field
+    if (lg.nv < 16u) {
+      vlo = (1u << (2u * lg.nv)) - 1u;
+      vhi = 0u;
+    } else if (lg.nv < 32u) {
+      vhi = (1u << (2u * (lg.nv - 16u))) - 1u;
+    }
+    vlo &= 0x55555555u;
+    vhi &= 0x55555555u;
 #pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i < cnt) {
-      uint32_t blk = warp * kWarpBlocks + i;
-      uint32_t off = __shfl_sync(kFull, my_off, blk);
-      uint32_t mu_bits = img_u32(sm.img, off);
-      float mu = __uint_as_float(mu_bits);
-      if (!((map >> blk) & 1u)) {
-        v[i] = make_float4(mu, mu, mu, mu);
-      } else {
-        uint32_t R = img_u8(sm.img, off + 4u);
-        uint32_t B = (R + 7u) >> 3;
-        uint32_t m = (blk == last_blk) ? jg.m_last : (uint32_t)kL;
-        uint32_t cb = (m + 3u) >> 2;
-        uint32_t code = (codes[i / 4] >> (8 * (i % 4))) & 0xffu;
-        int nv = (int)m - 4 * (int)lane;
-        nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
-        uint32_t nb0 = nv > 0 ? B - (code & 3u) : 0u;
-        uint32_t nb1 = nv > 1 ? B - ((code >> 2) & 3u) : 0u;
-        uint32_t nb2 = nv > 2 ? B - ((code >> 4) & 3u) : 0u;
-        uint32_t nb3 = nv > 3 ? B - ((code >> 6) & 3u) : 0u;
-        uint32_t T = (tp[i / 3] >> (10 * (i % 3))) & 0x3ffu;
-        uint32_t excl = ((incl[i / 3] >> (10 * (i % 3))) & 0x3ffu) - T;
-        // the lane's stored bytes as a little-endian 16-byte string
-        uint32_t so = off + 5u + cb + excl;
-        uint32_t wi = so >> 2, z = 8u * (so & 3u);
-        uint32_t A0 = sm.img[wi], A1 = sm.img[wi + 1], A2 = sm.img[wi + 2], A3 = sm.img[wi + 3], A4 = sm.img[wi + 4];
-        uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z),
-                 S3 = __funnelshift_r(A3, A4, z);
-        // peel the four elements off the front of the string
-        uint32_t r0 = S0;
-        uint32_t c0 = 8u * nb0;
-        uint32_t U0 = __funnelshift_rc(S0, S1, c0), U1 = __funnelshift_rc(S1, S2, c0), U2 = __funnelshift_rc(S2, S3, c0);
-        uint32_t r1 = U0;
-        uint32_t c1 = 8u * nb1;
-        uint32_t X0 = __funnelshift_rc(U0, U1, c1), X1 = __funnelshift_rc(U1, U2, c1);
-        uint32_t r2 = X0;
-        uint32_t r3 = __funnelshift_rc(X0, X1, 8u * nb2);
-        // stored bytes as a right-aligned big-endian value, and the byte mask they cover
-        uint32_t v0 = __funnelshift_rc(__byte_perm(r0, 0u, 0x0123), 0u, 32u - 8u * nb0);
-        uint32_t v1 = __funnelshift_rc(__byte_perm(r1, 0u, 0x0123), 0u, 32u - 8u * nb1);
-        uint32_t v2 = __funnelshift_rc(__byte_perm(r2, 0u, 0x0123), 0u, 32u - 8u * nb2);
-        uint32_t v3 = __funnelshift_rc(__byte_perm(r3, 0u, 0x0123), 0u, 32u - 8u * nb3);
-        uint32_t m0 = __funnelshift_rc(kFull, 0u, 32u - 8u * nb0);
-        uint32_t m1 = __funnelshift_rc(kFull, 0u, 32u - 8u * nb1);
-        uint32_t m2 = __funnelshift_rc(kFull, 0u, 32u - 8u * nb2);
-        uint32_t m3 = __funnelshift_rc(kFull, 0u, 32u - 8u * nb3);
-        // resolve the elided leading bytes inside the lane as if nothing came from the left ...
-        uint32_t l0 = v0;
-        uint32_t l1 = v1 | (l0 & ~m1);
-        uint32_t l2 = v2 | (l1 & ~m2);
-        uint32_t l3 = v3 | (l2 & ~m3);
-        uint32_t k0 = m0, k1 = k0 | m1, k2 = k1 | m2, k3 = k2 | m3;
-        // ... then carry the last code across lanes: bytes a lane does not cover come from its left
-        uint32_t cv = l3, cm = k3;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          uint32_t tv = __shfl_up_sync(kFull, cv, d);
-          uint32_t tm = __shfl_up_sync(kFull, cm, d);
-          cv = cv | (tv & ~cm);
-          cm = cm | tm;
-        }
-        uint32_t carry = __shfl_up_sync(kFull, cv, 1);
-        if (lane == 0) carry = 0u;
-        uint32_t q0 = l0 | (carry & ~k0), q1 = l1 | (carry & ~k1), q2 = l2 | (carry & ~k2), q3 = l3 | (carry & ~k3);
-        if (R == 32u) {
-          v[i] = make_float4(__uint_as_float(q0), __uint_as_float(q1), __uint_as_float(q2), __uint_as_float(q3));
+    for (uint32_t kb = 0; kb < 4; ++kb) {
+      if (kb < B) {
+        // values with lead <= kb store byte kb (counted from the most significant byte of the field)
+        uint32_t plo, phi;
+        if (kb == 0u) {
+          plo = ~(f0lo | f1lo), phi = ~(f0hi | f1hi);
+        } else if (kb == 1u) {
+          plo = ~f1lo, phi = ~f1hi;
+        } else if (kb == 2u) {
+          plo = ~(f0lo & f1lo), phi = ~(f0hi & f1hi);
         } else {
-          uint32_t sh = 32u - R;
-          v[i] = make_float4(__fadd_rn(__uint_as_float(q0 << sh), mu), __fadd_rn(__uint_as_float(q1 << sh), mu),
-                             __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
+          plo = phi = kFull;
+        }
+        plo &= vlo;
+        phi &= vhi;
+        if (plo | phi) {
+          uint32_t i = phi ? 16u + ((31u - (uint32_t)__clz(phi)) >> 1) : ((31u - (uint32_t)__clz(plo)) >> 1);
+          // bytes stored by the lane's values before value i
+          uint32_t mlo, mhi;
+          if (i < 16u) {
+            mlo = (1u << (2u * i)) - 1u;
+            mhi = 0u;
+          } else {
+            mlo = kFull;
+            mhi = (i == 16u) ? 0u : ((1u << (2u * (i - 16u))) - 1u);
+          }
+          uint32_t before = B * i - sum_fields2(code_lo & mlo, code_hi & mhi);
+          uint32_t lead_i = (i < 16u ? (code_lo >> (2u * i)) : (code_hi >> (2u * (i - 16u)))) & 3u;
+          uint32_t byte = img_u8(img, pos0 + before + (kb - lead_i));
+          uint32_t shift = 8u * (B - 1u - kb);
+          sval |= byte << shift;
+          smask |= 0xffu << shift;
         }
       }
+    }
+  }
+  // carry the summaries across the quad: what a lane does not store itself comes from its left
+  {
+    uint32_t tv = __shfl_up_sync(kFull, sval, 1), tm = __shfl_up_sync(kFull, smask, 1);
+    if (lg.t >= 1u) {
+      sval |= tv & ~smask;
+      smask |= tm;
+    }
+    tv = __shfl_up_sync(kFull, sval, 2);
+    tm = __shfl_up_sync(kFull, smask, 2);
+    if (lg.t >= 2u) {
+      sval |= tv & ~smask;
+      smask |= tm;
+    }
+  }
+  uint32_t prev = __shfl_up_sync(kFull, sval, 1);
+  if (lg.t == 0u) prev = 0u;
+
+  // the lane's 32 values
+  const float mu = (lg.m_blk != 0u) ? __uint_as_float(img_u32(img, boff)) : 0.0f;
+  if (!nonconst) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = make_float4(mu, mu, mu, mu);
+    return true;
+  }
+  const uint32_t sh = 32u - R;
+  uint32_t pos = pos0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t cb = ((j < 4) ? (code_lo >> (8 * j)) : (code_hi >> (8 * (j - 4)))) & 0xffu;
+    uint32_t nb0 = B - (cb & 3u), nb1 = B - ((cb >> 2) & 3u), nb2 = B - ((cb >> 4) & 3u), nb3 = B - ((cb >> 6) & 3u);
+    if (tail) {
+      if ((uint32_t)(4 * j + 0) >= lg.nv) nb0 = 0u;
+      if ((uint32_t)(4 * j + 1) >= lg.nv) nb1 = 0u;
+      if ((uint32_t)(4 * j + 2) >= lg.nv) nb2 = 0u;
+      if ((uint32_t)(4 * j + 3) >= lg.nv) nb3 = 0u;
+    }
+    // the quad's stored bytes as a little-endian 16-byte string
+    const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
+    const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3], A4 = img[wi + 4];
+    const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z),
+                   S3 = __funnelshift_r(A3, A4, z);
+    pos += nb0 + nb1 + nb2 + nb3;
+    // peel the four values off the front of the string
+    const uint32_t c0 = 8u * nb0, c1 = 8u * nb1, c2 = 8u * nb2;
+    const uint32_t U0 = __funnelshift_rc(S0, S1, c0), U1 = __funnelshift_rc(S1, S2, c0), U2 = __funnelshift_rc(S2, S3, c0);
+    const uint32_t X0 = __funnelshift_rc(U0, U1, c1), X1 = __funnelshift_rc(U1, U2, c1);
+    const uint32_t r3 = __funnelshift_rc(X0, X1, c2);
+    // stored bytes as a right-aligned big-endian value; the bytes not stored come from the predecessor
+    const uint32_t v0 = __funnelshift_rc(__byte_perm(S0, 0u, 0x0123), 0u, 32u - c0);
+    const uint32_t v1 = __funnelshift_rc(__byte_perm(U0, 0u, 0x0123), 0u, 32u - c1);
+    const uint32_t v2 = __funnelshift_rc(__byte_perm(X0, 0u, 0x0123), 0u, 32u - c2);
+    const uint32_t v3 = __funnelshift_rc(__byte_perm(r3, 0u, 0x0123), 0u, 32u - 8u * nb3);
+    const uint32_t q0 = v0 | (prev & ~__funnelshift_rc(kFull, 0u, 32u - c0));
+    const uint32_t q1 = v1 | (q0 & ~__funnelshift_rc(kFull, 0u, 32u - c1));
+    const uint32_t q2 = v2 | (q1 & ~__funnelshift_rc(kFull, 0u, 32u - c2));
+    const uint32_t q3 = v3 | (q2 & ~__funnelshift_rc(kFull, 0u, 32u - 8u * nb3));
+    prev = q3;
+    if (R == 32u) {
+      v[j] = make_float4(__uint_as_float(q0), __uint_as_float(q1), __uint_as_float(q2), __uint_as_float(q3));
+    } else {
+      v[j] = make_float4(__fadd_rn(__uint_as_float(q0 << sh), mu), __fadd_rn(__uint_as_float(q1 << sh), mu),
+                         __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
     }
   }
   return true;
 }
 
-// Store the blocks a warp decoded (or summed): one 128-bit store per lane and block.
-__device__ __forceinline__ void store_blocks(float* out, const JobGeom& jg, uint32_t g, const float4 (&v)[kWarpBlocks]) {
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    uint32_t gblk = g * kGroupBlocks + warp * kWarpBlocks + i;
-    if (gblk < jg.nb) {
-      float* p = out + (uint64_t)gblk * kL + 4u * lane;
-      uint32_t m = (gblk == jg.nb - 1) ? jg.m_last : (uint32_t)kL;
-      if (4u * lane + 4u <= m) {
-        __stcs(reinterpret_cast<float4*>(p), v[i]);
-      } else {
-        if (4u * lane + 0u < m) p[0] = v[i].x;
-        if (4u * lane + 1u < m) p[1] = v[i].y;
-        if (4u * lane + 2u < m) p[2] = v[i].z;
-      }
-    }
-  }
+// Stage group payload words [a, a+gw) of the stream into the image.
+__device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
+  const uint32_t* src = sv.words + (sv.base >> 2) + sv.a;
+  for (uint32_t j = threadIdx.x; j < sv.gw; j += kThreads) sm.img[j] = __ldcs(src + j);
 }
 
 // ---------------------------------------------------------------------------------------------------
 // kernels
 // ---------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) compress_kernel(const __grid_constant__ EncodeBatch b) {
-  __shared__ __align__(16) EncSmem sm;
+__global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
+  Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
+  uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
   const JobGeom jg = job_geom(b.n, b.chunk_len, y);
   uint8_t* sout = b.sout + (uint64_t)y * b.s_stride;
@@ -688,15 +881,21 @@ __global__ void __launch_bounds__(kThreads) compress_kernel(const __grid_constan
   if (g >= jg.G) return;
   const uint32_t rank = (uint32_t)((y + (uint32_t)b.rot) % (uint32_t)b.P);
   const float* x = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
-  float4 v[kWarpBlocks];
-  load_blocks(x, jg, g, v);
+  const LaneGeom lg = lane_geom(jg, g);
+  load_rows(rows, x, jg, g);
   zero_image(sm.img);
-  encode_group(sm, v, b, jg, g, y, sout);
+  if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
+  __syncthreads();
+  float4 v[8];
+  const float4* slice = reinterpret_cast<const float4*>(rows + threadIdx.x * kSliceBytes);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = slice[j];
+  encode_group(sm, rows, v, lg, b, jg, g, y, sout);
 }
 
-__global__ void __launch_bounds__(kThreads) reduce_kernel(const __grid_constant__ EncodeBatch b) {
-  __shared__ __align__(16) EncSmem sm;
-  __shared__ __align__(16) DecSmem dm;
+__global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
+  Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
+  uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
   const JobGeom jg = job_geom(b.n, b.chunk_len, y);
   uint8_t* sout = b.sout + (uint64_t)y * b.s_stride;
@@ -707,36 +906,54 @@ __global__ void __launch_bounds__(kThreads) reduce_kernel(const __grid_constant_
   if (g >= jg.G) return;
   const uint32_t rank = (uint32_t)((y + (uint32_t)b.rot) % (uint32_t)b.P);
   const float* local = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
-  float4 loc[kWarpBlocks];
-  load_blocks(local, jg, g, loc);
-  zero_image(sm.img);
+  const LaneGeom lg = lane_geom(jg, g);
+  load_rows(rows, local, jg, g);
+  if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
+
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   StreamView sv;
-  float4 v[kWarpBlocks];
+  float4 v[8];
   bool ok = open_group(sin, in_bytes, jg, g, sv);
-  if (ok) ok = decode_group(dm, sv, jg, g, v);
+  if (ok) {
+    stage_payload(sm, sv);
+    __syncthreads();
+    ok = decode_group(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v);
+  }
   if (!ok) {
     // a corrupt input: report it, and keep the look-back chain alive with a poisoned entry
     if (threadIdx.x == 0) {
       raise(b.status, kErrCorrupt);
-      st_relaxed_u64(b.tile_state + (uint64_t)y * b.tiles_per_job + g, pack_state(b.epoch, kFlagPoison, 0));
+      uint64_t* A = b.tile_state + (uint64_t)y * b.state_stride;
+      st_relaxed_u64(&A[g], pack_state(b.epoch, kFlagPoison, 0));
+      if ((g & 31u) == 31u || g == jg.G - 1u)
+        st_relaxed_u64(&A[b.tiles_per_job + (g >> 5)], pack_state(b.epoch, kFlagPoison, 0));
     }
     return;
   }
+  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
 #pragma unroll
-  for (int i = 0; i < kWarpBlocks; ++i) {
-    v[i].x = __fadd_rn(v[i].x, loc[i].x);
-    v[i].y = __fadd_rn(v[i].y, loc[i].y);
-    v[i].z = __fadd_rn(v[i].z, loc[i].z);
-    v[i].w = __fadd_rn(v[i].w, loc[i].w);
+  for (int j = 0; j < 8; ++j) {
+    float4 l = slice[j];
+    v[j].x = __fadd_rn(v[j].x, l.x);
+    v[j].y = __fadd_rn(v[j].y, l.y);
+    v[j].z = __fadd_rn(v[j].z, l.z);
+    v[j].w = __fadd_rn(v[j].w, l.w);
   }
-  if (b.sum_out) store_blocks(b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g, v);
-  encode_group(sm, v, b, jg, g, y, sout);
+  __syncthreads();  // every thread is done reading the incoming image
+  zero_image(sm.img);
+  write_slice(rows, v);  // the general encode path re-reads the values from the slice
+  if (b.sum_out) {
+    __syncthreads();
+    store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
+    __syncthreads();  // the slices are about to be reused for staging
+  }
+  encode_group(sm, rows, v, lg, b, jg, g, y, sout);
 }
 
-__global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant__ DecodeBatch b) {
-  __shared__ __align__(16) DecSmem dm;
+__global__ void __launch_bounds__(kThreads, 6) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b) {
+  Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
+  uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y, z = blockIdx.z;
   if (b.skip_mode == 1 && z == (y + (uint32_t)b.P - 1u) % (uint32_t)b.P) return;
   if (b.skip_mode == 2 && z == 0u) return;
@@ -746,27 +963,61 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const __grid_constant_
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   float* out = b.scatter ? b.out + (uint64_t)y * b.out_rank_stride : b.out + (uint64_t)z * b.out_rank_stride + jg.lo;
+  const LaneGeom lg = lane_geom(jg, g);
   StreamView sv;
-  float4 v[kWarpBlocks];
+  float4 v[8];
   bool ok = open_group(sin, in_bytes, jg, g, sv);
-  if (ok) ok = decode_group(dm, sv, jg, g, v);
+  if (ok) {
+    stage_payload(sm, sv);
+    __syncthreads();
+    ok = decode_group(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v);
+  }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
     return;
   }
-  store_blocks(out, jg, g, v);
+  write_slice(rows, v);
+  __syncthreads();
+  store_rows(rows, out, jg, g);
 }
 
 }  // namespace
 
-void launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
-  compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, 0, s>>>(b);
+namespace {
+constexpr int kSmemBytes = kCtlBytes + kRowsBytes;
+
+// Per device: opt in to the dynamic shared-memory size once.
+bool g_ready[64];
+bool device_ready() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  if (!g_ready[dev]) {
+    if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(ccoll_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+      return false;
+    g_ready[dev] = true;
+  }
+  return true;
 }
-void launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
-  reduce_kernel<<<dim3(groups_x, jobs, 1), kThreads, 0, s>>>(b);
+}  // namespace
+
+// Groups wait (bounded) on the sizes of earlier groups of their job; CTAs are issued in blockIdx order
+// (x fastest), so the CTAs a group depends on are always resident or finished.
+bool launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
+  if (!device_ready()) return false;
+  ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+  return true;
 }
-void launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
-  decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, 0, s>>>(b);
+bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
+  if (!device_ready()) return false;
+  ccoll_reduce_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+  return true;
+}
+bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
+  if (!device_ready()) return false;
+  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemBytes, s>>>(b);
+  return true;
 }
 
 }  // namespace ccoll

@@ -29,11 +29,11 @@ constexpr int kImgWords = kMaxGroupBytes / 4 + 24;                    // image +
 // status codes mirrored from ccoll.h
 constexpr uint32_t kErrCapacity = 3, kErrCorrupt = 4, kErrTimeout = 5;
 
-// Look-back state word: [epoch:32][flag:2][value:30].  A word whose epoch differs from the launch's epoch
-// is "not written yet", so the state array never needs clearing between launches.
-constexpr uint32_t kFlagAggregate = 1, kFlagPrefix = 2, kFlagPoison = 3;
+// Size word of a group / super-group: [epoch:32][flag:2][value:30].  A word whose epoch differs from the
+// launch's epoch is "not written yet", so the array never needs clearing between launches.
+constexpr uint32_t kFlagAggregate = 1, kFlagPoison = 3;
 constexpr uint32_t kValueMask = (1u << 30) - 1;
-constexpr uint32_t kSpinLimit = 1u << 21;  // polls (each followed by a short sleep) before giving up
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls (each followed by a short sleep) before giving up
 
 // A family of encode jobs (one job per blockIdx.y): job y covers values [y*C, min(n, (y+1)*C)) of the
 // buffer of virtual rank (y + rot) mod P.
@@ -54,8 +54,9 @@ struct EncodeBatch {
   uint64_t sum_rank_stride;
   uint64_t* moved;          // nullable: += moved_mult * stream bytes of every job
   uint32_t moved_mult;
-  uint64_t* tile_state;     // look-back words, job y at tile_state + y*tiles_per_job
+  uint64_t* tile_state;     // size words: job y has A[tiles_per_job] then SA[ceil(tiles_per_job/32)] at y*state_stride
   uint32_t tiles_per_job;
+  uint32_t state_stride;
   uint32_t epoch;
   uint32_t* status;         // sticky error word
   float eb;
@@ -78,8 +79,9 @@ struct DecodeBatch {
   uint32_t* status;
 };
 
-void launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
-void launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
-void launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s);
+// Each returns false if the device could not be set up (the launch was not attempted).
+bool launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
+bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
+bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s);
 
 }  // namespace ccoll
