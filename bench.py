@@ -42,6 +42,20 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def max_over_ranks(value, dist, device="cuda"):
+    """The slowest rank sets the time of a multi-rank measurement."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(world, bytes_per_rank, ms):
+    """GB/s over all ranks: replicas do the same work each, so the job's bytes are world x the rank's."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons (read-only NVML queries) while the timed region runs."""
 
@@ -277,15 +291,11 @@ def main():
     sync_all()
     clocks = sampler.stop()
     assert B.ccoll_get_status() == B.OK
-    total_ms = t_begin.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), dist)
     ms_per_step = total_ms / args.steps
     call_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(5)]
     bytes_per_step = 5 * 4 * n
-    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_throughput(world, bytes_per_step, ms_per_step)
 
     # ---- rooflines of the three kernels (each of calls 1-3 is exactly one launch) ----
     peak, peak_kind = measured_peaks()
@@ -336,12 +346,8 @@ def main():
     for _ in range(e2e_steps):
         e2e_step()
     sync_all()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * bytes_per_step / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": 2 * 4 * n,
+    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps, dist)
+    e2e = {"value": whole_job_throughput(world, bytes_per_step, e2e_s * 1e3), "unit": "GB/s", "h2d_bytes_per_step": 2 * 4 * n,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_s * 1e3}
 
     if rank == 0:

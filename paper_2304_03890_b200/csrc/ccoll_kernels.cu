@@ -554,11 +554,7 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
   }
 
   // place of the group in the stream
-#ifdef CCOLL_EXP_NOPREFIX
-  if (threadIdx.x == 0) sm.prefix = g * words;
-#else
   find_prefix(sm, A, SA, g, jg.G, words, b.epoch, b.status);
-#endif
   __syncthreads();
   const uint32_t prefix = sm.prefix;
   if (sm.fail) return;
@@ -570,17 +566,10 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
     return;
   }
   {
-    // coalesced copy-out: single words up to the first 16-byte boundary of the stream, then 128-bit stores
+    // coalesced copy-out: consecutive lanes move consecutive words (conflict-free shared reads, full
+    // 128-byte lines per warp store)
     uint32_t* dst = out32 + (base >> 2) + prefix;
-    const uint32_t head = min(words, (4u - (((base >> 2) + prefix) & 3u)) & 3u);
-    if (tid < head) dst[tid] = sm.img[tid];
-    const uint32_t nvec = (words - head) >> 2;
-    uint4* dst4 = reinterpret_cast<uint4*>(dst + head);
-    const uint32_t* src = sm.img + head;
-    for (uint32_t i = tid; i < nvec; i += kThreads)
-      dst4[i] = make_uint4(src[4u * i], src[4u * i + 1u], src[4u * i + 2u], src[4u * i + 3u]);
-    const uint32_t done = head + 4u * nvec;
-    if (tid < words - done) dst[done + tid] = sm.img[done + tid];
+    for (uint32_t j = tid; j < words; j += kThreads) __stcs(dst + j, sm.img[j]);
   }
   if (tid == 0) {
     out32[8 + g] = prefix;             // dir[g]

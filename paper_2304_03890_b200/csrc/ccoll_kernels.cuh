@@ -1,12 +1,12 @@
 // ccoll_kernels.cuh — sm_100a kernels of the C-Coll hot path: block classify + encode + size scan and
 // compaction (compress), the parallel decoder, and the fused decompress-add-recompress ring round.
 //
-// Work decomposition (all three kernels): one CTA of 4 warps owns one GROUP of 32 blocks (4096 values);
-// warp w owns blocks 8w .. 8w+7 of it; within a block lane l owns elements 4l .. 4l+3, i.e. exactly one
-// 128-bit coalesced load / store.  Everything a block needs from its neighbours' lanes travels by warp
-// shuffles or warp reductions; the variable-length bytes are assembled in registers, placed into a
+// Work decomposition (all three kernels): one CTA of 128 threads owns one GROUP of 32 blocks (4096 values).
+// Thread t owns slice t = 32 consecutive values, so the four lanes 4b .. 4b+3 share block b.  Per-value
+// work runs serially inside a lane; what must cross lanes (min/max, the predecessor code, byte offsets)
+// is a two-step shuffle inside the quad.  Variable-length bytes are staged per lane, copied once into a
 // shared-memory image of the group's payload, and leave the SM as coalesced word stores at the offset
-// found by a decoupled look-back over the groups' sizes.
+// that the two-level sum of the earlier groups' sizes yields.
 #pragma once
 
 #include <cstdint>
@@ -20,7 +20,6 @@ constexpr int kGroupBlocks = 32;           // blocks per group
 constexpr int kGroupValues = kL * kGroupBlocks;
 constexpr int kWarps = 4;
 constexpr int kThreads = 32 * kWarps;
-constexpr int kWarpBlocks = kGroupBlocks / kWarps;  // 8 blocks per warp
 constexpr int kHeaderBytes = 32;
 constexpr int kMaxRecord = 5 + kL / 4 + 4 * kL;                       // 549
 constexpr int kMaxGroupBytes = 2 * kGroupBlocks + kGroupBlocks * kMaxRecord;  // 17632 (a multiple of 4)

@@ -1,0 +1,43 @@
+"""The C-ABI library builds, loads without a GPU and exports every function include/ccoll.h declares."""
+import ctypes
+import os
+import re
+
+from paper_2304_03890_b200 import binding as B
+from paper_2304_03890_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ccoll.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ccoll_[a-z_]+)\s*\(", text)))
+
+
+def test_header_and_library_agree():
+    names = declared_functions()
+    assert set(names) == set(B.EXPORTS)
+    lib = ctypes.CDLL(build.build())
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_host_only_entry_points():
+    # these need no device
+    assert B.ccoll_compress_bound(0) == 32 + 4 + 15
+    assert B.ccoll_compress_bound(4096) == 32 + 8 + 4 + 15 + (64 + 32 * 549 + 3)
+    assert B.ccoll_compress_bound(1000, 64) == 0            # unsupported block length
+    assert B.ccoll_chunk_len(25557032, 16) == 1597440
+    assert B.ccoll_chunk_len(100, 8) == 128
+    assert B.ccoll_workspace_bytes(1 << 20, 128, 1) > 0
+    assert B.ccoll_workspace_bytes(1 << 24, 128, 8) > B.ccoll_workspace_bytes(1 << 24, 128, 1)
+    assert B.ccoll_workspace_bytes(1 << 20, 128, 5000) == 0  # more virtual ranks than supported
+
+
+def test_bound_and_chunk_rule_match_the_oracle():
+    from oracle import ccz
+    for n in (0, 1, 127, 128, 4096, 4097, 1 << 20, 25557032):
+        assert B.ccoll_compress_bound(n) == ccz.compress_bound(n)
+        for P in (1, 3, 8, 16, 32):
+            assert B.ccoll_chunk_len(n, P) == ccz.chunk_len(n, P)
