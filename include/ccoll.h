@@ -133,6 +133,34 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
 int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n,
                     float abs_err_bound, uint32_t block_len, int mode, uint64_t* chunk_bytes, void* stream);
 
+/* ccoll_compress for callers that cannot give the library scratch memory.  (No counterpart in the paper: it
+ * is a packaging of ccoll_compress, not a step of the method.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested any more — a communication runtime
+ * whose host application has already handed the whole GPU to its own memory pool, a plug-in called from
+ * inside someone else's step where cudaMalloc may fail, or would stall every stream of the device while it
+ * runs.  Such a caller cannot create the workspace that ccoll_set_workspace wants.  Here the kernel's scratch
+ * (one 8-byte size word per 4096 values and one per 131072 values) is a fixed array inside the library's
+ * device image instead; this function calls no cudaMalloc / cudaFree and no routine that allocates, and it
+ * does not use or need the registered workspace.
+ *
+ *   in, n, abs_err_bound, block_len, out, out_bytes, stream   exactly as for ccoll_compress; the stream it
+ *              writes is byte-identical to ccoll_compress's.
+ *   status     REQUIRED device u32 owned by the caller, zero before the call: receives (by atomic max) a
+ *              ccoll_status_t if the kernel meets an error only the GPU can see.  It takes the place of the
+ *              workspace's status word; ccoll_get_status does not report on this call.
+ * Limits and rules:
+ *   - n <= CCOLL_NOALLOC_MAX_VALUES (64 Mi values = 256 MiB of fp32); more returns CCOLL_ERR_CAPACITY and
+ *     nothing is launched.  The array costs every GPU that loads the library about 136 KB until exit.
+ *   - The first call on a device looks up the array's device address (and does the kernels' one-time
+ *     set-up); make that first call outside any stream capture.
+ *   - All calls on one device share the one array, which keeps what the last call wrote.  Nothing has to be
+ *     cleared by the caller (entries are tagged per call), but two calls that overlap on the GPU — different
+ *     streams, no ordering between them — race on it and corrupt each other's output.  Order them. */
+#define CCOLL_NOALLOC_MAX_VALUES ((size_t)1 << 26)
+int ccoll_compress_noalloc(const float* in, size_t n, float abs_err_bound, uint32_t block_len, void* out,
+                           uint64_t* out_bytes, uint32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -17,7 +17,7 @@ _NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CAPACITY", 4: "CORRUP
 
 EXPORTS = ("ccoll_compress_bound", "ccoll_chunk_len", "ccoll_workspace_bytes", "ccoll_set_workspace",
            "ccoll_get_status", "ccoll_compress", "ccoll_decompress", "ccoll_reduce_step", "ccoll_allreduce_sim",
-           "ccoll_bcast_sim")
+           "ccoll_bcast_sim", "ccoll_compress_noalloc")
 
 _lib = None
 
@@ -55,6 +55,8 @@ def lib():
     L.ccoll_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp, vp]
     L.ccoll_bcast_sim.restype = i32
     L.ccoll_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp, vp]
+    L.ccoll_compress_noalloc.restype = i32
+    L.ccoll_compress_noalloc.argtypes = [vp, sz, f32, u32, vp, vp, vp, vp]
     _lib = L
     return L
 
@@ -144,6 +146,13 @@ def ccoll_bcast_sim(root, out, out_rank_stride, P, eb, mode=BCAST, chunk_bytes=N
                     stream=None):
     _check(lib().ccoll_bcast_sim(_ptr(root), _ptr(out), out_rank_stride, P, root.numel(), eb, block_len, mode,
                                  _ptr(chunk_bytes), _stream(stream)), "ccoll_bcast_sim")
+
+
+def ccoll_compress_noalloc(x, eb, out, out_bytes, status, block_len=BLOCK_LEN, stream=None):
+    """ccoll_compress without a workspace: the scratch is a fixed array inside the library (see ccoll.h).
+    `status` is a zeroed uint32/int32 CUDA tensor of one element that receives device-side errors."""
+    _check(lib().ccoll_compress_noalloc(_ptr(x), x.numel(), eb, block_len, _ptr(out), _ptr(out_bytes), _ptr(status),
+                                        _stream(stream)), "ccoll_compress_noalloc")
 
 
 # ---- conveniences for tests and examples (allocation with torch, still no arithmetic) -----------------------

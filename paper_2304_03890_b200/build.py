@@ -8,7 +8,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = [os.path.join(CSRC, f) for f in ("ccoll_kernels.cu", "ccoll_api.cu")]
+SOURCES = [os.path.join(CSRC, f) for f in ("ccoll_kernels.cu", "ccoll_api.cu", "ccoll_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "ccoll_kernels.cuh"), os.path.join(os.path.dirname(HERE), "include", "ccoll.h")]
 LIB = os.path.join(HERE, "libccoll.so")
 

@@ -1,0 +1,62 @@
+"""ccoll_compress_noalloc — the entry point for callers that cannot allocate device memory (an application
+that has given the whole GPU to its own pool, a plug-in that must not call cudaMalloc inside someone else's
+step): its scratch is a fixed array inside the library.  It must write the very stream ccoll_compress writes,
+call after call, although every call finds the previous call's leftovers in that array.
+
+Collected last on purpose (file name), so a run that stops at the first failure has run everything else."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2304_03890_b200 import binding as B
+from paper_2304_03890_b200 import fields
+
+pytestmark = pytest.mark.gpu
+
+
+def reference_stream(x, eb):
+    """The existing entry point (workspace-based), through the C ABI."""
+    return B.compress(x, eb)
+
+
+def noalloc_stream(x, eb):
+    out = torch.empty(B.ccoll_compress_bound(x.numel()), dtype=torch.uint8, device="cuda")
+    nbytes = torch.zeros(1, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = B.lib().ccoll_compress_noalloc(ctypes.c_void_p(x.data_ptr()), x.numel(), eb, 128,
+                                        ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(nbytes.data_ptr()),
+                                        ctypes.c_void_p(status.data_ptr()),
+                                        ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    assert rc == B.OK
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.OK
+    return out[: int(nbytes.item())]
+
+
+def test_two_calls_in_a_row_match_the_workspace_entry_point():
+    # a large field first, then a smaller ragged one: the second call sees the first call's size words
+    big = fields.config2(device="cuda", shape=(128, 128, 256), sigma=8.0)
+    small = fields.config1(device="cuda", n=4096 * 37 + 1000 + 3)
+    for cfg in (big, small, big):
+        x, eb = cfg["x"], float(cfg["eb"])
+        got = noalloc_stream(x, eb)
+        want = reference_stream(x, eb)
+        assert got.numel() == want.numel()
+        assert torch.equal(got, want)           # bit-exact, the bar of every parity test here
+
+
+def test_empty_input_and_size_limit():
+    x = torch.zeros(0, device="cuda")
+    assert noalloc_stream(x, 1e-3).numel() == 48
+    L = B.lib()
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    too_many = (1 << 26) + 1
+    rc = L.ccoll_compress_noalloc(ctypes.c_void_p(dummy.data_ptr()), too_many, 1e-3, 128,
+                                  ctypes.c_void_p(dummy.data_ptr()), None, ctypes.c_void_p(st.data_ptr()), None)
+    assert rc == B.ERR_CAPACITY                 # refused before anything is launched
+    rc = L.ccoll_compress_noalloc(ctypes.c_void_p(dummy.data_ptr()), 16, 1e-3, 128,
+                                  ctypes.c_void_p(dummy.data_ptr()), None, None, None)
+    assert rc == B.ERR_INVALID_ARG              # the status word is required
