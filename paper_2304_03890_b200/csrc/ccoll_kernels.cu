@@ -18,6 +18,19 @@
 #include "ccoll_kernels.cuh"
 
 namespace ccoll {
+#ifdef CCOLL_TIMELINE  // development aid: per-CTA phase timestamps (never compiled into the shipped library)
+__device__ unsigned long long g_timeline[8192 * 8];
+#define TL(slot)                                                                   \
+  do {                                                                             \
+    if (threadIdx.x == 0 && blockIdx.x < 8192 && blockIdx.y == 0 && blockIdx.z == 0) { \
+      unsigned long long t_;                                                       \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                       \
+      g_timeline[blockIdx.x * 8 + (slot)] = t_;                                    \
+    }                                                                              \
+  } while (0)
+#else
+#define TL(slot) do {} while (0)
+#endif
 namespace {
 
 constexpr uint32_t kFull = 0xffffffffu;
@@ -857,7 +870,10 @@ __device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
 // ---------------------------------------------------------------------------------------------------
 // kernels
 // ---------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
+#ifndef CCOLL_EXP_CTAS
+#define CCOLL_EXP_CTAS 6
+#endif
+__global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
@@ -940,9 +956,11 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   encode_group(sm, rows, v, lg, b, jg, g, y, sout);
 }
 
-__global__ void __launch_bounds__(kThreads, 6) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b) {
-  Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
-  uint8_t* rows = dyn_smem + kCtlBytes;
+// The incoming image is dead once every lane holds its decoded values in registers, so the rows the values
+// leave through reuse the same shared memory: 18 KB per CTA, which lets 9 CTAs share an SM.
+__global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b) {
+  Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);  // only sm.img is used here
+  uint8_t* rows = dyn_smem;                        // aliases sm.img
   const uint32_t g = blockIdx.x, y = blockIdx.y, z = blockIdx.z;
   if (b.skip_mode == 1 && z == (y + (uint32_t)b.P - 1u) % (uint32_t)b.P) return;
   if (b.skip_mode == 2 && z == 0u) return;
@@ -955,25 +973,33 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_decode_kernel(const __grid_
   const LaneGeom lg = lane_geom(jg, g);
   StreamView sv;
   float4 v[8];
+  TL(0);
   bool ok = open_group(sin, in_bytes, jg, g, sv);
+  TL(1);
   if (ok) {
     stage_payload(sm, sv);
     __syncthreads();
+    TL(2);
     ok = decode_group(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v);
   }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
     return;
   }
+  TL(3);
+  __syncthreads();  // every lane is done reading the image
   write_slice(rows, v);
   __syncthreads();
+  TL(4);
   store_rows(rows, out, jg, g);
+  TL(5);
 }
 
 }  // namespace
 
 namespace {
 constexpr int kSmemBytes = kCtlBytes + kRowsBytes;
+constexpr int kSmemDecode = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
 
 // Per device: opt in to the dynamic shared-memory size once.
 bool g_ready[64];
@@ -983,7 +1009,7 @@ bool device_ready() {
   if (!g_ready[dev]) {
     if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDecode) != cudaSuccess)
       return false;
     g_ready[dev] = true;
   }
@@ -1005,8 +1031,13 @@ bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaS
 }
 bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
   if (!device_ready()) return false;
-  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemBytes, s>>>(b);
+  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b);
   return true;
 }
 
+#ifdef CCOLL_TIMELINE
+extern "C" int ccoll_debug_timeline(unsigned long long* host, size_t count) {
+  return (int)cudaMemcpyFromSymbol(host, g_timeline, count * sizeof(unsigned long long));
+}
+#endif
 }  // namespace ccoll
