@@ -32,6 +32,15 @@ SHAPE = (512, 512, 256)
 SIGMA = 8.0
 P_SIM = 8
 METRIC = "compress / decompress / fused reduce-step GB/s (fp32 input) and % of B200 HBM peak"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of each kernel on the
+# 256x512x256 field of the same recipe (33,554,432 values; profiles/kernels_256x512x256_four_lanes_per_block.md),
+# expressed per value: DRAM traffic grows in proportion to the values processed, so a full-size launch is
+# this figure times its value count.  (Writes that are still in L2 when the kernel ends are not in it.)
+NCU_DRAM_BYTES_PER_VALUE = {
+    "ccoll_compress_kernel": (134.33e6 + 8.64e6) / 33554432,
+    "ccoll_decode_kernel": (58.71e6 + 76.01e6) / 33554432,
+    "ccoll_reduce_kernel": (193.06e6 + 150.80e6) / 33554432,
+}
 
 
 def measured_peaks():
@@ -309,7 +318,9 @@ def main():
     for name, ms in zip(("ccoll_compress_kernel", "ccoll_decode_kernel", "ccoll_reduce_kernel"), call_ms[:3]):
         ach = alg[name] / (ms * 1e-3) / 1e9
         roofs[name] = {"bound": "hbm", "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                       "frac": ach / peak, "traffic": None, "algorithmic_bytes": alg[name], "ms": ms,
+                       "frac": ach / peak, "traffic": NCU_DRAM_BYTES_PER_VALUE[name] * n,
+                       "traffic_source": "ncu capture at 33.5M values, scaled by value count",
+                       "algorithmic_bytes": alg[name], "ms": ms,
                        "input_GBps": 4 * n / (ms * 1e-3) / 1e9}
     dominant = "ccoll_reduce_kernel"
     roofline = dict(roofs[dominant], kernel=dominant)

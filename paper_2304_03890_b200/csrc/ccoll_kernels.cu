@@ -510,7 +510,7 @@ __device__ __forceinline__ void find_prefix(Smem& sm, uint64_t* A, uint64_t* SA,
 // barrier inside) before the call.
 __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v)[8], const LaneGeom& lg,
                                              const EncodeBatch& b, const JobGeom& jg, uint32_t g, uint32_t y,
-                                             uint8_t* sout) {
+                                             uint8_t* sout, bool values_not_in_slice) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   uint32_t* slice = reinterpret_cast<uint32_t*>(rows + tid * kSliceBytes);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
@@ -521,10 +521,16 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
   if (lg.t == 0u) prev = 0u;
   uint32_t T = 0u, code_lo = 0u, code_hi = 0u;
   if (p.R != 0u) {
-    if (tail || p.lossless)
+    if (tail || p.lossless) {
+      if (values_not_in_slice) {  // the general path re-reads the values from the lane's own slice
+        float4* own = reinterpret_cast<float4*>(slice);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) own[j] = v[j];
+      }
       emit_lane_slow(slice, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
-    else
+    } else {
       emit_lane_fast(slice, v, p, prev, T, code_lo, code_hi);
+    }
   }
   uint32_t total;
   const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
@@ -639,6 +645,7 @@ struct StreamView {
   const uint32_t* words;  // the stream as 32-bit words
   uint32_t G, base;       // groups, payload_base
   uint32_t a, gw, map;    // first payload word of the group, its length in words, its bitmap
+  uint32_t pw;            // payload words of the whole stream
 };
 
 // Validate the header and the directory entries of group g.  Every thread of the CTA reads the same words
@@ -663,6 +670,7 @@ __device__ __forceinline__ bool open_group(const uint8_t* sin, uint64_t in_bytes
   if (nblk < 32u && (sv.map >> nblk) != 0u) return false;
   sv.a = a;
   sv.gw = e - a;
+  sv.pw = (uint32_t)pw;
   return true;
 }
 
@@ -677,7 +685,7 @@ __device__ __forceinline__ uint32_t sum_fields2(uint32_t lo, uint32_t hi) {
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
                                              float4 (&v)[8]) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
-  const uint32_t* img = sm.img;
+  const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
 
   // offsets of the 32 records: lane b looks at block b
@@ -820,6 +828,37 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   }
   const uint32_t sh = 32u - R;
   uint32_t pos = pos0;
+  if (!tail && R <= 24u) {
+    // Fast path: complete slice, field of at most 3 bytes.  Shifts by computed amounts are multiplications
+    // by a power of two (FMA pipe) where the power serves twice: m = 2^(8*stored bytes) extracts the stored
+    // bytes (umulhi) and -m masks the bytes that are kept from the predecessor.
+    const uint32_t c8B = 8u * B;
+    const uint32_t msh = 1u << sh;  // q << sh == q * 2^sh
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t cb = ((j < 4) ? (code_lo >> (8 * j)) : (code_hi >> (8 * (j - 4)))) & 0xffu;
+      const uint32_t c0 = c8B - 8u * (cb & 3u), c1 = c8B - 8u * ((cb >> 2) & 3u), c2 = c8B - 8u * ((cb >> 4) & 3u),
+                     c3 = c8B - 8u * (cb >> 6);
+      const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
+      const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3];
+      // at most 12 bytes per quad here: three words of string are enough
+      const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z);
+      pos += (c0 + c1 + c2 + c3) >> 3;
+      const uint32_t U0 = __funnelshift_r(S0, S1, c0), U1 = __funnelshift_r(S1, S2, c0);
+      const uint32_t X0 = __funnelshift_r(U0, U1, c1);
+      const uint32_t X1 = __funnelshift_r(U1, S2 >> c0, c1);
+      const uint32_t r3 = __funnelshift_r(X0, X1, c2);
+      const uint32_t m0 = 1u << c0, m1 = 1u << c1, m2 = 1u << c2, m3 = 1u << c3;
+      const uint32_t q0 = __umulhi(__byte_perm(S0, 0u, 0x0123), m0) | (prev & (0u - m0));
+      const uint32_t q1 = __umulhi(__byte_perm(U0, 0u, 0x0123), m1) | (q0 & (0u - m1));
+      const uint32_t q2 = __umulhi(__byte_perm(X0, 0u, 0x0123), m2) | (q1 & (0u - m2));
+      const uint32_t q3 = __umulhi(__byte_perm(r3, 0u, 0x0123), m3) | (q2 & (0u - m3));
+      prev = q3;
+      v[j] = make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
+                         __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu));
+    }
+    return true;
+  }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const uint32_t cb = ((j < 4) ? (code_lo >> (8 * j)) : (code_hi >> (8 * (j - 4)))) & 0xffu;
@@ -861,10 +900,36 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   return true;
 }
 
-// Stage group payload words [a, a+gw) of the stream into the image.
+// Stage group payload words [a, a+gw) of the stream into the image.  All of a thread's loads are issued
+// before the first store (a rolled loop would pay one memory round trip per iteration), and they are 128
+// bits wide: the copy starts at the 16-byte boundary at or below word a, so payload word j lands at
+// sm.img[(a & 3) + j] — decode_group reads the image through that shifted origin.
+constexpr int kStageRounds = (kMaxGroupBytes / 4 + 3 + 4 * kThreads - 1) / (4 * kThreads);  // 9
 __device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
-  const uint32_t* src = sv.words + (sv.base >> 2) + sv.a;
-  for (uint32_t j = threadIdx.x; j < sv.gw; j += kThreads) sm.img[j] = __ldcs(src + j);
+  const uint32_t shift = sv.a & 3u;
+  const uint32_t n_words = sv.gw + shift;             // words to bring in, from the aligned start
+  const uint32_t* src = sv.words + (sv.base >> 2) + (sv.a - shift);
+  const uint32_t avail = sv.pw - (sv.a - shift);      // payload words from the aligned start to the stream's end
+  uint4 t[kStageRounds];
+#pragma unroll
+  for (int r = 0; r < kStageRounds; ++r) {
+    const uint32_t w = 4u * ((uint32_t)r * kThreads + threadIdx.x);
+    t[r] = make_uint4(0u, 0u, 0u, 0u);
+    if (w < n_words) {
+      if (w + 4u <= avail) {
+        t[r] = __ldcs(reinterpret_cast<const uint4*>(src + w));
+      } else {  // the very end of the stream: never read past it
+        if (w + 0u < avail) t[r].x = __ldcs(src + w + 0u);
+        if (w + 1u < avail) t[r].y = __ldcs(src + w + 1u);
+        if (w + 2u < avail) t[r].z = __ldcs(src + w + 2u);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kStageRounds; ++r) {
+    const uint32_t w = 4u * ((uint32_t)r * kThreads + threadIdx.x);
+    if (w < n_words) *reinterpret_cast<uint4*>(&sm.img[w]) = t[r];
+  }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -895,7 +960,7 @@ __global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kerne
   const float4* slice = reinterpret_cast<const float4*>(rows + threadIdx.x * kSliceBytes);
 #pragma unroll
   for (int j = 0; j < 8; ++j) v[j] = slice[j];
-  encode_group(sm, rows, v, lg, b, jg, g, y, sout);
+  encode_group(sm, rows, v, lg, b, jg, g, y, sout, false);
 }
 
 __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
@@ -947,13 +1012,13 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   }
   __syncthreads();  // every thread is done reading the incoming image
   zero_image(sm.img);
-  write_slice(rows, v);  // the general encode path re-reads the values from the slice
   if (b.sum_out) {
+    write_slice(rows, v);
     __syncthreads();
     store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
     __syncthreads();  // the slices are about to be reused for staging
   }
-  encode_group(sm, rows, v, lg, b, jg, g, y, sout);
+  encode_group(sm, rows, v, lg, b, jg, g, y, sout, b.sum_out == nullptr);
 }
 
 // The incoming image is dead once every lane holds its decoded values in registers, so the rows the values
