@@ -19,13 +19,13 @@
 
 namespace ccoll {
 #ifdef CCOLL_TIMELINE  // development aid: per-CTA phase timestamps (never compiled into the shipped library)
-__device__ unsigned long long g_timeline[8192 * 8];
+__device__ unsigned long long g_timeline[8192 * 16];
 #define TL(slot)                                                                   \
   do {                                                                             \
     if (threadIdx.x == 0 && blockIdx.x < 8192 && blockIdx.y == 0 && blockIdx.z == 0) { \
       unsigned long long t_;                                                       \
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                       \
-      g_timeline[blockIdx.x * 8 + (slot)] = t_;                                    \
+      g_timeline[blockIdx.x * 16 + (slot)] = t_;                                    \
     }                                                                              \
   } while (0)
 #else
@@ -236,25 +236,17 @@ struct Plan {
   bool lossless;
 };
 
-template <bool kTail>
-__device__ __forceinline__ Plan plan_block(float4 (&v)[8], const LaneGeom& lg, uint32_t lane, float eb, int eb_exp) {
-  if (kTail) {
-    // values past the end of the data are replaced by the block's first value: they cannot change min or max
-    float f = __shfl_sync(kFull, v[0].x, lane & ~3u);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if ((uint32_t)(4 * j + 0) >= lg.nv) v[j].x = f;
-      if ((uint32_t)(4 * j + 1) >= lg.nv) v[j].y = f;
-      if ((uint32_t)(4 * j + 2) >= lg.nv) v[j].z = f;
-      if ((uint32_t)(4 * j + 3) >= lg.nv) v[j].w = f;
-    }
-  }
-  float mx = max3_nan(max_nan(v[0].x, v[0].y), v[0].z, v[0].w);
-  float mn = min3_nan(min_nan(v[0].x, v[0].y), v[0].z, v[0].w);
-#pragma unroll
+// The loops over a lane's eight quads read the values from the lane's slice and are only unrolled twice:
+// fully unrolled on register arrays the fused kernel outgrew the 32 KB instruction cache (84 % hit rate).
+__device__ __forceinline__ Plan plan_block(const float4* x4, const LaneGeom& lg, float eb, int eb_exp) {
+  float4 q = x4[0];
+  float mx = max3_nan(max_nan(q.x, q.y), q.z, q.w);
+  float mn = min3_nan(min_nan(q.x, q.y), q.z, q.w);
+#pragma unroll 2
   for (int j = 1; j < 8; ++j) {
-    mx = max3_nan(max3_nan(mx, v[j].x, v[j].y), v[j].z, v[j].w);
-    mn = min3_nan(min3_nan(mn, v[j].x, v[j].y), v[j].z, v[j].w);
+    q = x4[j];
+    mx = max3_nan(max3_nan(mx, q.x, q.y), q.z, q.w);
+    mn = min3_nan(min3_nan(mn, q.x, q.y), q.z, q.w);
   }
   mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 1));
   mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 1));
@@ -345,32 +337,35 @@ __device__ __forceinline__ void finish_stage(Stage& st) {
   st.wp[1] = 0u;        // and a zero word behind it for the realigning copy
 }
 
-// Fast path: all 32 values valid, block not lossless, values in registers.
-__device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const float4 (&v)[8], const Plan& p, uint32_t prev,
-                                               uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+// Fast path: all 32 values valid, block not lossless.  Values are read from the slice quad by quad; the
+// staged bytes overwrite the slice in place, which is safe because quad j is read before anything is
+// written at or behind its position.
+__device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const Plan& p, uint32_t prev, uint32_t& T_out,
+                                               uint32_t& code_lo, uint32_t& code_hi) {
   const uint32_t fix = (p.B == 4u) ? 1u : 0u;
   const uint32_t cadj = (4u - p.B) * 85u;
   const float mu = p.mu;
   const uint32_t sh = p.sh;
   Stage st = {slice, 0u, 0u, 0u};
-  code_lo = code_hi = 0u;
-#pragma unroll
+  uint64_t codes = 0ull;
+  const float4* x4 = reinterpret_cast<const float4*>(slice);
+#pragma unroll 2
   for (int j = 0; j < 8; ++j) {
-    const uint32_t q0 = __float_as_uint(__fsub_rn(v[j].x, mu)) >> sh, q1 = __float_as_uint(__fsub_rn(v[j].y, mu)) >> sh,
-                   q2 = __float_as_uint(__fsub_rn(v[j].z, mu)) >> sh, q3 = __float_as_uint(__fsub_rn(v[j].w, mu)) >> sh;
+    const float4 x = x4[j];
+    const uint32_t q0 = __float_as_uint(__fsub_rn(x.x, mu)) >> sh, q1 = __float_as_uint(__fsub_rn(x.y, mu)) >> sh,
+                   q2 = __float_as_uint(__fsub_rn(x.z, mu)) >> sh, q3 = __float_as_uint(__fsub_rn(x.w, mu)) >> sh;
     const uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
                    sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
     prev = q3;
     // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field
     const uint32_t cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) >> 3) - cadj;
-    if (j < 4)
-      code_lo |= cb << (8 * j);
-    else
-      code_hi |= cb << (8 * (j - 4));
+    codes |= (uint64_t)cb << (8 * j);
     append_quad(st, q0, q1, q2, q3, sa0, sa1, sa2, sa3);
   }
   finish_stage(st);
   T_out = st.Tb >> 3;
+  code_lo = (uint32_t)codes;
+  code_hi = (uint32_t)(codes >> 32);
 }
 
 // General path (ragged slices, lossless blocks): rolled loop over the quads, values re-read from the slice.
@@ -508,29 +503,30 @@ __device__ __forceinline__ void find_prefix(Smem& sm, uint64_t* A, uint64_t* SA,
 // Encode the group whose values the threads hold in v[] (32 per thread), build its payload image, find its
 // place in the stream and copy it out.  The image must have been zeroed (and that made visible by the
 // barrier inside) before the call.
-__device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v)[8], const LaneGeom& lg,
-                                             const EncodeBatch& b, const JobGeom& jg, uint32_t g, uint32_t y,
-                                             uint8_t* sout, bool values_not_in_slice) {
+__device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const LaneGeom& lg, const EncodeBatch& b,
+                                             const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   uint32_t* slice = reinterpret_cast<uint32_t*>(rows + tid * kSliceBytes);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
 
-  Plan p = tail ? plan_block<true>(v, lg, lane, b.eb, b.eb_exp) : plan_block<false>(v, lg, lane, b.eb, b.eb_exp);
+  if (tail && lg.nv < (uint32_t)kSliceVals) {
+    // Ragged slice (rare): values past the end of the data are replaced by the block's first value, so that
+    // they cannot change min or max.  (The first value of block b is the first value of slice 4b.)
+    const float f = *reinterpret_cast<const float*>(rows + (tid & ~3u) * kSliceBytes);
+    float* x = reinterpret_cast<float*>(slice);
+    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) x[i] = f;
+  }
+  if (tail) __syncwarp();
+  Plan p = plan_block(reinterpret_cast<const float4*>(slice), lg, b.eb, b.eb_exp);
   // code of the value just before this lane's first one (0 at the start of a block)
-  uint32_t prev = __shfl_up_sync(kFull, code_of(v[7].w, p), 1);
+  uint32_t prev = __shfl_up_sync(kFull, code_of(reinterpret_cast<const float*>(slice)[kSliceVals - 1], p), 1);
   if (lg.t == 0u) prev = 0u;
   uint32_t T = 0u, code_lo = 0u, code_hi = 0u;
   if (p.R != 0u) {
-    if (tail || p.lossless) {
-      if (values_not_in_slice) {  // the general path re-reads the values from the lane's own slice
-        float4* own = reinterpret_cast<float4*>(slice);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) own[j] = v[j];
-      }
+    if (tail || p.lossless)
       emit_lane_slow(slice, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
-    } else {
-      emit_lane_fast(slice, v, p, prev, T, code_lo, code_hi);
-    }
+    else
+      emit_lane_fast(slice, p, prev, T, code_lo, code_hi);
   }
   uint32_t total;
   const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
@@ -540,6 +536,7 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
     sm.blk_R[lg.blk] = p.R;
   }
   __syncthreads();  // sizes visible; also: image zero-fill and all staging done
+  TL(4);
 
   // every warp derives the offsets of all 32 records (cheap, and saves a barrier)
   const uint32_t sz_l = sm.blk_size[lane];
@@ -573,8 +570,11 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
   }
 
   // place of the group in the stream
+  TL(5);
   find_prefix(sm, A, SA, g, jg.G, words, b.epoch, b.status);
+  TL(11);
   __syncthreads();
+  TL(6);
   const uint32_t prefix = sm.prefix;
   if (sm.fail) return;
   const uint32_t base = payload_base(jg.G);
@@ -588,12 +588,15 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, float4 (&v
     // coalesced copy-out: consecutive lanes move consecutive words (conflict-free shared reads, full
     // 128-byte lines per warp store)
     uint32_t* dst = out32 + (base >> 2) + prefix;
+    TL(8);
     for (uint32_t j = tid; j < words; j += kThreads) __stcs(dst + j, sm.img[j]);
+    TL(9);
   }
   if (tid == 0) {
     out32[8 + g] = prefix;             // dir[g]
     out32[8 + jg.G + 1 + g] = bitmap;  // bitmap[g]
   }
+  TL(10);
   if (g == 0 && tid >= 32 && tid < 32 + 4) {
     // static part of the header and the zero pad between the bitmap and the payload
     uint32_t t = tid - 32;
@@ -680,10 +683,55 @@ __device__ __forceinline__ uint32_t sum_fields2(uint32_t lo, uint32_t hi) {
          2u * (uint32_t)(__popc(lo & 0xaaaaaaaau) + __popc(hi & 0xaaaaaaaau));
 }
 
+// One quad of the general decode path: any field width, lossless blocks, ragged slices (nvq = valid values
+// of the quad).  Out of line on purpose (rare, and it keeps the kernels' hot code small).
+struct DecodeCursor {
+  uint32_t pos;   // image offset of the next stored byte
+  uint32_t prev;  // code of the previous value
+};
+__device__ __noinline__ float4 decode_quad_generic(const uint32_t* img, DecodeCursor& cur, uint32_t cb, uint32_t R,
+                                                   float mu, uint32_t nvq) {
+  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
+  uint32_t nb0 = B - (cb & 3u), nb1 = B - ((cb >> 2) & 3u), nb2 = B - ((cb >> 4) & 3u), nb3 = B - ((cb >> 6) & 3u);
+  if (nvq < 1u) nb0 = 0u;
+  if (nvq < 2u) nb1 = 0u;
+  if (nvq < 3u) nb2 = 0u;
+  if (nvq < 4u) nb3 = 0u;
+  // the quad's stored bytes as a little-endian 16-byte string
+  const uint32_t wi = cur.pos >> 2, z = 8u * (cur.pos & 3u);
+  const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3], A4 = img[wi + 4];
+  const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z),
+                 S3 = __funnelshift_r(A3, A4, z);
+  cur.pos += nb0 + nb1 + nb2 + nb3;
+  // peel the four values off the front of the string
+  const uint32_t c0 = 8u * nb0, c1 = 8u * nb1, c2 = 8u * nb2, c3 = 8u * nb3;
+  const uint32_t U0 = __funnelshift_rc(S0, S1, c0), U1 = __funnelshift_rc(S1, S2, c0), U2 = __funnelshift_rc(S2, S3, c0);
+  const uint32_t X0 = __funnelshift_rc(U0, U1, c1), X1 = __funnelshift_rc(U1, U2, c1);
+  const uint32_t r3 = __funnelshift_rc(X0, X1, c2);
+  // stored bytes as a right-aligned big-endian value; the bytes not stored come from the predecessor
+  const uint32_t v0 = __funnelshift_rc(__byte_perm(S0, 0u, 0x0123), 0u, 32u - c0);
+  const uint32_t v1 = __funnelshift_rc(__byte_perm(U0, 0u, 0x0123), 0u, 32u - c1);
+  const uint32_t v2 = __funnelshift_rc(__byte_perm(X0, 0u, 0x0123), 0u, 32u - c2);
+  const uint32_t v3 = __funnelshift_rc(__byte_perm(r3, 0u, 0x0123), 0u, 32u - c3);
+  const uint32_t q0 = v0 | (cur.prev & ~__funnelshift_rc(kFull, 0u, 32u - c0));
+  const uint32_t q1 = v1 | (q0 & ~__funnelshift_rc(kFull, 0u, 32u - c1));
+  const uint32_t q2 = v2 | (q1 & ~__funnelshift_rc(kFull, 0u, 32u - c2));
+  const uint32_t q3 = v3 | (q2 & ~__funnelshift_rc(kFull, 0u, 32u - c3));
+  cur.prev = q3;
+  if (R == 32u) return make_float4(__uint_as_float(q0), __uint_as_float(q1), __uint_as_float(q2), __uint_as_float(q3));
+  return make_float4(__fadd_rn(__uint_as_float(q0 << sh), mu), __fadd_rn(__uint_as_float(q1 << sh), mu),
+                     __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
+}
+
 // Decode the lane's 32 values of group g into v[].  Returns false (for the whole CTA) on a corrupt group.
 // The group's payload must already be staged in sm.img (and visible).  nblk = blocks in the group.
+// kToSlice = false: the values are returned in v[] (fully unrolled loops).  kToSlice = true (fused reduce):
+// each decoded quad is ADDED to the quad of local values waiting in the lane's slice and the sum is written
+// back there; the loops are then unrolled only twice, which keeps the fused kernel inside the instruction
+// cache.
+template <bool kToSlice>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8]) {
+                                             float4 (&v)[8], float4* slice4) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
@@ -754,51 +802,24 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   const uint32_t pos0 = boff + 5u + cbytes + excl;  // image offset of the lane's first stored byte
   uint32_t sval = 0u, smask = 0u;
   if (nonconst && lg.nv != 0u) {
-    const uint32_t f0lo = code_lo & 0x55555555u, f1lo = (code_lo >> 1) & 0x55555555u;
-    const uint32_t f0hi = code_hi & 0x55555555u, f1hi = (code_hi >> 1) & 0x55555555u;
-    uint32_t vlo = 0x55555555u, vhi = 0x55555555u;  // valid values of the lane, one bit per 2-bit field
-    if (lg.nv < 16u) {
-      vlo = (1u << (2u * lg.nv)) - 1u;
-      vhi = 0u;
-    } else if (lg.nv < 32u) {
-      vhi = (1u << (2u * (lg.nv - 16u))) - 1u;
-    }
-    vlo &= 0x55555555u;
-    vhi &= 0x55555555u;
-#pragma unroll
-    for (uint32_t kb = 0; kb < 4; ++kb) {
-      if (kb < B) {
-        // values with lead <= kb store byte kb (counted from the most significant byte of the field)
-        uint32_t plo, phi;
-        if (kb == 0u) {
-          plo = ~(f0lo | f1lo), phi = ~(f0hi | f1hi);
-        } else if (kb == 1u) {
-          plo = ~f1lo, phi = ~f1hi;
-        } else if (kb == 2u) {
-          plo = ~(f0lo & f1lo), phi = ~(f0hi & f1hi);
-        } else {
-          plo = phi = kFull;
-        }
-        plo &= vlo;
-        phi &= vhi;
-        if (plo | phi) {
-          uint32_t i = phi ? 16u + ((31u - (uint32_t)__clz(phi)) >> 1) : ((31u - (uint32_t)__clz(plo)) >> 1);
-          // bytes stored by the lane's values before value i
-          uint32_t mlo, mhi;
-          if (i < 16u) {
-            mlo = (1u << (2u * i)) - 1u;
-            mhi = 0u;
-          } else {
-            mlo = kFull;
-            mhi = (i == 16u) ? 0u : ((1u << (2u * (i - 16u))) - 1u);
-          }
-          uint32_t before = B * i - sum_fields2(code_lo & mlo, code_hi & mhi);
-          uint32_t lead_i = (i < 16u ? (code_lo >> (2u * i)) : (code_hi >> (2u * (i - 16u)))) & 3u;
-          uint32_t byte = img_u8(img, pos0 + before + (kb - lead_i));
-          uint32_t shift = 8u * (B - 1u - kb);
-          sval |= byte << shift;
-          smask |= 0xffu << shift;
-        }
+    const uint64_t codes = ((uint64_t)code_hi << 32) | code_lo;
+    const uint64_t kOdd = 0x5555555555555555ull;  // one marker bit per 2-bit field
+    const uint64_t f0 = codes & kOdd, f1 = (codes >> 1) & kOdd;
+    const uint64_t valid = (lg.nv < 32u ? ((1ull << (2u * lg.nv)) - 1ull) : ~0ull) & kOdd;
+#pragma unroll 1
+    for (uint32_t kb = 0; kb < B; ++kb) {
+      // values with lead <= kb store byte kb (counted from the most significant byte of the field)
+      uint64_t pm = kb == 0u ? ~(f0 | f1) : (kb == 1u ? ~f1 : (kb == 2u ? ~(f0 & f1) : ~0ull));
+      pm &= valid;
+      if (pm) {
+        const uint32_t i = (63u - (uint32_t)__clzll((long long)pm)) >> 1;  // the last such value
+        const uint64_t below = codes & ((1ull << (2u * i)) - 1ull);        // codes of the values before it
+        const uint32_t lead_sum = (uint32_t)__popcll(below & kOdd) + 2u * (uint32_t)__popcll(below & (kOdd << 1));
+        const uint32_t lead_i = (uint32_t)(codes >> (2u * i)) & 3u;
+        const uint32_t byte = img_u8(img, pos0 + (B * i - lead_sum) + (kb - lead_i));
+        const uint32_t shift = 8u * (B - 1u - kb);
+        sval |= byte << shift;
+        smask |= 0xffu << shift;
       }
     }
   }
@@ -821,11 +842,21 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
 
   // the lane's 32 values
   const float mu = (lg.m_blk != 0u) ? __uint_as_float(img_u32(img, boff)) : 0.0f;
+  constexpr int kUnroll = kToSlice ? 2 : 8;
+  auto put = [&](int j, const float4& r) {
+    if (kToSlice) {
+      const float4 a = slice4[j];
+      slice4[j] = make_float4(__fadd_rn(r.x, a.x), __fadd_rn(r.y, a.y), __fadd_rn(r.z, a.z), __fadd_rn(r.w, a.w));
+    } else {
+      v[j] = r;
+    }
+  };
   if (!nonconst) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = make_float4(mu, mu, mu, mu);
+#pragma unroll kUnroll
+    for (int j = 0; j < 8; ++j) put(j, make_float4(mu, mu, mu, mu));
     return true;
   }
+  const uint64_t codes = ((uint64_t)code_hi << 32) | code_lo;
   const uint32_t sh = 32u - R;
   uint32_t pos = pos0;
   if (!tail && R <= 24u) {
@@ -834,9 +865,9 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
     // bytes (umulhi) and -m masks the bytes that are kept from the predecessor.
     const uint32_t c8B = 8u * B;
     const uint32_t msh = 1u << sh;  // q << sh == q * 2^sh
-#pragma unroll
+#pragma unroll kUnroll
     for (int j = 0; j < 8; ++j) {
-      const uint32_t cb = ((j < 4) ? (code_lo >> (8 * j)) : (code_hi >> (8 * (j - 4)))) & 0xffu;
+      const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
       const uint32_t c0 = c8B - 8u * (cb & 3u), c1 = c8B - 8u * ((cb >> 2) & 3u), c2 = c8B - 8u * ((cb >> 4) & 3u),
                      c3 = c8B - 8u * (cb >> 6);
       const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
@@ -854,48 +885,18 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
       const uint32_t q2 = __umulhi(__byte_perm(X0, 0u, 0x0123), m2) | (q1 & (0u - m2));
       const uint32_t q3 = __umulhi(__byte_perm(r3, 0u, 0x0123), m3) | (q2 & (0u - m3));
       prev = q3;
-      v[j] = make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
-                         __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu));
+      put(j, make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
+                         __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu)));
     }
     return true;
   }
-#pragma unroll
+  // General path (ragged slice, 4-byte field, lossless block): one out-of-line call per quad.
+  DecodeCursor cur = {pos0, prev};
+#pragma unroll kUnroll
   for (int j = 0; j < 8; ++j) {
-    const uint32_t cb = ((j < 4) ? (code_lo >> (8 * j)) : (code_hi >> (8 * (j - 4)))) & 0xffu;
-    uint32_t nb0 = B - (cb & 3u), nb1 = B - ((cb >> 2) & 3u), nb2 = B - ((cb >> 4) & 3u), nb3 = B - ((cb >> 6) & 3u);
-    if (tail) {
-      if ((uint32_t)(4 * j + 0) >= lg.nv) nb0 = 0u;
-      if ((uint32_t)(4 * j + 1) >= lg.nv) nb1 = 0u;
-      if ((uint32_t)(4 * j + 2) >= lg.nv) nb2 = 0u;
-      if ((uint32_t)(4 * j + 3) >= lg.nv) nb3 = 0u;
-    }
-    // the quad's stored bytes as a little-endian 16-byte string
-    const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
-    const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3], A4 = img[wi + 4];
-    const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z),
-                   S3 = __funnelshift_r(A3, A4, z);
-    pos += nb0 + nb1 + nb2 + nb3;
-    // peel the four values off the front of the string
-    const uint32_t c0 = 8u * nb0, c1 = 8u * nb1, c2 = 8u * nb2;
-    const uint32_t U0 = __funnelshift_rc(S0, S1, c0), U1 = __funnelshift_rc(S1, S2, c0), U2 = __funnelshift_rc(S2, S3, c0);
-    const uint32_t X0 = __funnelshift_rc(U0, U1, c1), X1 = __funnelshift_rc(U1, U2, c1);
-    const uint32_t r3 = __funnelshift_rc(X0, X1, c2);
-    // stored bytes as a right-aligned big-endian value; the bytes not stored come from the predecessor
-    const uint32_t v0 = __funnelshift_rc(__byte_perm(S0, 0u, 0x0123), 0u, 32u - c0);
-    const uint32_t v1 = __funnelshift_rc(__byte_perm(U0, 0u, 0x0123), 0u, 32u - c1);
-    const uint32_t v2 = __funnelshift_rc(__byte_perm(X0, 0u, 0x0123), 0u, 32u - c2);
-    const uint32_t v3 = __funnelshift_rc(__byte_perm(r3, 0u, 0x0123), 0u, 32u - 8u * nb3);
-    const uint32_t q0 = v0 | (prev & ~__funnelshift_rc(kFull, 0u, 32u - c0));
-    const uint32_t q1 = v1 | (q0 & ~__funnelshift_rc(kFull, 0u, 32u - c1));
-    const uint32_t q2 = v2 | (q1 & ~__funnelshift_rc(kFull, 0u, 32u - c2));
-    const uint32_t q3 = v3 | (q2 & ~__funnelshift_rc(kFull, 0u, 32u - 8u * nb3));
-    prev = q3;
-    if (R == 32u) {
-      v[j] = make_float4(__uint_as_float(q0), __uint_as_float(q1), __uint_as_float(q2), __uint_as_float(q3));
-    } else {
-      v[j] = make_float4(__fadd_rn(__uint_as_float(q0 << sh), mu), __fadd_rn(__uint_as_float(q1 << sh), mu),
-                         __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
-    }
+    const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
+    const uint32_t done = 4u * (uint32_t)j;
+    put(j, decode_quad_generic(img, cur, cb, R, mu, lg.nv > done ? lg.nv - done : 0u));
   }
   return true;
 }
@@ -956,11 +957,7 @@ __global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kerne
   zero_image(sm.img);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
   __syncthreads();
-  float4 v[8];
-  const float4* slice = reinterpret_cast<const float4*>(rows + threadIdx.x * kSliceBytes);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) v[j] = slice[j];
-  encode_group(sm, rows, v, lg, b, jg, g, y, sout, false);
+  encode_group(sm, rows, lg, b, jg, g, y, sout);
 }
 
 __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
@@ -977,19 +974,24 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const uint32_t rank = (uint32_t)((y + (uint32_t)b.rot) % (uint32_t)b.P);
   const float* local = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
+  TL(0);
   load_rows(rows, local, jg, g);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
 
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   StreamView sv;
-  float4 v[8];
+  float4 unused[8];
+  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
   bool ok = open_group(sin, in_bytes, jg, g, sv);
   if (ok) {
     stage_payload(sm, sv);
-    __syncthreads();
-    ok = decode_group(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v);
+    __syncthreads();  // the image and the local values in the rows are complete
+    TL(1);
+    // decoded + local, one rounded add per value, left in the lane's slice
+    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice);
   }
+  TL(2);
   if (!ok) {
     // a corrupt input: report it, and keep the look-back chain alive with a poisoned entry
     if (threadIdx.x == 0) {
@@ -1001,24 +1003,15 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     }
     return;
   }
-  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    float4 l = slice[j];
-    v[j].x = __fadd_rn(v[j].x, l.x);
-    v[j].y = __fadd_rn(v[j].y, l.y);
-    v[j].z = __fadd_rn(v[j].z, l.z);
-    v[j].w = __fadd_rn(v[j].w, l.w);
-  }
-  __syncthreads();  // every thread is done reading the incoming image
+  __syncthreads();  // every thread is done reading the incoming image (and has written its sums)
   zero_image(sm.img);
   if (b.sum_out) {
-    write_slice(rows, v);
-    __syncthreads();
     store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
     __syncthreads();  // the slices are about to be reused for staging
   }
-  encode_group(sm, rows, v, lg, b, jg, g, y, sout, b.sum_out == nullptr);
+  TL(3);
+  encode_group(sm, rows, lg, b, jg, g, y, sout);
+  TL(7);
 }
 
 // The incoming image is dead once every lane holds its decoded values in registers, so the rows the values
@@ -1045,7 +1038,7 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
     stage_payload(sm, sv);
     __syncthreads();
     TL(2);
-    ok = decode_group(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v);
+    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr);
   }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
