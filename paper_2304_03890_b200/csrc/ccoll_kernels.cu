@@ -172,6 +172,13 @@ __device__ __forceinline__ void zero_image(uint32_t* img) {  // a barrier must f
 // Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
 // (128-bit streaming loads) and scatters them into the padded slices; in round r thread tid moves the
 // float4 number r*128 + tid of the group.  A __syncthreads must follow before the slices are read.
+// Ask L2 for the fp32 values of a group that a later CTA will load (one 128-byte line per thread).  Issued by
+// the CTA that currently occupies the SM slot that later CTA will get, so its loads find the data in L2.
+__device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg, uint32_t g) {
+  if (g >= jg.G) return;
+  const uint64_t first = (uint64_t)g * kGroupValues + 32u * threadIdx.x;
+  if (first < jg.len) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + first));
+}
 __device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
   const uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
@@ -901,6 +908,15 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   return true;
 }
 
+// Ask L2 for the payload of group gp of the stream (a later CTA will stage it).  The two directory words
+// are loaded by the caller early (dir_a, dir_e); nothing is validated here, a prefetch cannot fault.
+__device__ __forceinline__ void prefetch_payload(const StreamView& sv, uint32_t dir_a, uint32_t dir_e) {
+  if (dir_e <= dir_a || dir_e - dir_a > (uint32_t)kMaxGroupBytes / 4u || dir_e > sv.pw) return;
+  const uint8_t* base = reinterpret_cast<const uint8_t*>(sv.words) + sv.base;
+  for (uint32_t off = 4u * dir_a + 128u * threadIdx.x; off < 4u * dir_e; off += 128u * kThreads)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+}
+
 // Stage group payload words [a, a+gw) of the stream into the image.  All of a thread's loads are issued
 // before the first store (a rolled loop would pay one memory round trip per iteration), and they are 128
 // bits wide: the copy starts at the 16-byte boundary at or below word a, so payload word j lands at
@@ -954,6 +970,7 @@ __global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kerne
   const float* x = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
   load_rows(rows, x, jg, g);
+  prefetch_group(x, jg, g + b.prefetch_distance);
   zero_image(sm.img);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
   __syncthreads();
@@ -976,6 +993,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const LaneGeom lg = lane_geom(jg, g);
   TL(0);
   load_rows(rows, local, jg, g);
+  prefetch_group(local, jg, g + b.prefetch_distance);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
 
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
@@ -984,8 +1002,14 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   float4 unused[8];
   float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
   bool ok = open_group(sin, in_bytes, jg, g, sv);
+  uint32_t nxt_a = 0u, nxt_e = 0u;  // directory entries of the group that will take over this SM slot
+  if (ok && g + b.prefetch_distance < jg.G) {
+    nxt_a = __ldg(sv.words + 8 + g + b.prefetch_distance);
+    nxt_e = __ldg(sv.words + 8 + g + b.prefetch_distance + 1);
+  }
   if (ok) {
     stage_payload(sm, sv);
+    prefetch_payload(sv, nxt_a, nxt_e);
     __syncthreads();  // the image and the local values in the rows are complete
     TL(1);
     // decoded + local, one rounded add per value, left in the lane's slice
@@ -1034,8 +1058,14 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   TL(0);
   bool ok = open_group(sin, in_bytes, jg, g, sv);
   TL(1);
+  uint32_t nxt_a = 0u, nxt_e = 0u;  // directory entries of the group that will take over this SM slot
+  if (ok && g + b.prefetch_distance < jg.G) {
+    nxt_a = __ldg(sv.words + 8 + g + b.prefetch_distance);
+    nxt_e = __ldg(sv.words + 8 + g + b.prefetch_distance + 1);
+  }
   if (ok) {
     stage_payload(sm, sv);
+    prefetch_payload(sv, nxt_a, nxt_e);
     __syncthreads();
     TL(2);
     ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr);
@@ -1059,16 +1089,25 @@ namespace {
 constexpr int kSmemBytes = kCtlBytes + kRowsBytes;
 constexpr int kSmemDecode = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
 
-// Per device: opt in to the dynamic shared-memory size once.
+// Per device: opt in to the dynamic shared-memory size once, and learn how many CTAs of the encoding kernels
+// are resident at a time (the distance of their L2 prefetch).
 bool g_ready[64];
+uint32_t g_slots[64], g_slots_decode[64];
 bool device_ready() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
   if (!g_ready[dev]) {
+    int sms = 0, per_sm = 0;
     if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDecode) != cudaSuccess)
+        cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDecode) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_compress_kernel, kThreads, kSmemBytes) != cudaSuccess)
       return false;
+    g_slots[dev] = (uint32_t)(sms * (per_sm > 0 ? per_sm : 1));
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_decode_kernel, kThreads, kSmemDecode) != cudaSuccess)
+      return false;
+    g_slots_decode[dev] = (uint32_t)(sms * (per_sm > 0 ? per_sm : 1));
     g_ready[dev] = true;
   }
   return true;
@@ -1077,18 +1116,33 @@ bool device_ready() {
 
 // Groups wait (bounded) on the sizes of earlier groups of their job; CTAs are issued in blockIdx order
 // (x fastest), so the CTAs a group depends on are always resident or finished.
-bool launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
+static EncodeBatch with_prefetch(const EncodeBatch& b, uint32_t jobs) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  EncodeBatch c = b;
+  // CTAs are issued x-fastest: with one job the slot of group g is taken over by group g + slots
+  c.prefetch_distance = jobs == 1 ? g_slots[dev] : (g_slots[dev] + jobs - 1) / jobs;
+  return c;
+}
+bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
+  const EncodeBatch b = with_prefetch(b0, jobs);
   ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
   return true;
 }
-bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
+bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
+  const EncodeBatch b = with_prefetch(b0, jobs);
   ccoll_reduce_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
   return true;
 }
-bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
+bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
   if (!device_ready()) return false;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  DecodeBatch b = b0;
+  const uint32_t streams = jobs * ranks;  // CTAs are issued x-fastest over (group, stream, rank)
+  b.prefetch_distance = streams == 1 ? g_slots_decode[dev] : (g_slots_decode[dev] + streams - 1) / streams;
   ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b);
   return true;
 }

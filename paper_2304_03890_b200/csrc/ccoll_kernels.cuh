@@ -61,6 +61,7 @@ struct EncodeBatch {
   uint32_t tiles_per_job;
   uint32_t state_stride;
   uint32_t epoch;
+  uint32_t prefetch_distance;  // groups ahead whose values a CTA asks L2 for (set by the launcher)
   uint32_t* status;         // sticky error word
   float eb;
   int eb_exp;               // biased exponent field of eb
@@ -79,6 +80,7 @@ struct DecodeBatch {
   int P;
   int skip_mode;   // 0 none; 1 skip rank z == (y-1) mod P (the chunk's owner); 2 skip z == 0; 3 skip y == 0
   int scatter;     // 1: job y writes at out + y*out_rank_stride; 0: at out + z*out_rank_stride + y*C
+  uint32_t prefetch_distance;  // groups ahead whose payload a CTA asks L2 for (set by the launcher)
   uint32_t* status;
 };
 
