@@ -152,3 +152,27 @@ def test_config4_scatter_and_bcast_full():
         for c in range(1, P):
             assert torch.equal(bc[r, c * C: (c + 1) * C], sc[c])
         assert float((bc[r, :C].double() - root[:C].double()).abs().max()) <= eb
+
+
+def test_maximum_stream_size():
+    """n = CCOLL_MAX_VALUES (2^29 values, 2 GiB of fp32): one stream of 131072 groups; one more value is refused."""
+    n = 1 << 29
+    g = torch.Generator(device="cuda")
+    g.manual_seed(fields.seed_for(9))
+    # a cheap smooth-ish signal at full length: random walk per 4096-value group on top of a slow ramp
+    x = torch.randn(n, generator=g, device="cuda").mul_(1e-2)
+    x = x.view(-1, GROUP).cumsum(dim=1).view(-1).contiguous()
+    eb = 1e-2
+    stream = B.compress(x, eb)
+    G = n // GROUP
+    check_sampled_groups(x, stream, eb, sample_groups(G, 12, seed=3))
+    dec = B.decompress(stream, n)
+    step = 1 << 26
+    for a in range(0, n, step):            # in pieces: the fp64 temporaries would not fit otherwise
+        assert float((dec[a:a + step].double() - x[a:a + step].double()).abs().max()) <= eb
+    del dec, stream
+    out = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.CcollError) as e:
+        B.lib()  # noqa: keep the library loaded
+        B._check(B.lib().ccoll_compress(x.data_ptr(), n + 1, eb, 128, out.data_ptr(), None, None), "ccoll_compress")
+    assert e.value.code == B.ERR_UNSUPPORTED

@@ -241,3 +241,23 @@ def test_argument_checks():
         B.ccoll_compress(x[1:], 1e-3, out)       # misaligned
     assert e.value.code == B.ERR_INVALID_ARG
     assert L.ccoll_compress(None, 8, 1e-3, 128, None, None, None) == B.ERR_INVALID_ARG
+
+
+def test_many_virtual_ranks():
+    """P = 1024 (the most the replays accept): one 128-value block per chunk, some chunks empty."""
+    P = 1024
+    rng = np.random.default_rng(12)
+    n = 128 * 1000 + 40                     # chunk = 128 values; chunks 1001.. are empty
+    root = np.cumsum(rng.normal(0, 0.01, n)).astype(np.float32)[: n // 4 * 4]
+    eb = 1e-3
+    ref, ref_cb = ccz.bcast_sim(root, P, eb, mode=1)
+    got, cb = B.bcast_sim(dev(root), P, eb, mode=B.SCATTER)
+    assert np.array_equal(cb.cpu().numpy().astype(np.uint64), ref_cb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes()
+    x = rng.normal(0, 1, (P, 128 * 20)).astype(np.float32)   # chunk = 128 values for ranks 0..19, rest empty
+    ref, ref_moved = ccz.allreduce_sim(x, eb)
+    got, moved = B.allreduce_sim(dev(x), eb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
+    with pytest.raises(B.CcollError) as e:
+        B.ccoll_bcast_sim(dev(root), torch.empty(8, device="cuda"), 0, 1025, eb)
+    assert e.value.code == B.ERR_INVALID_ARG
