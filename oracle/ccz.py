@@ -9,6 +9,7 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_CORRUPT = 0, 1, 3, 4
 BLOCK_CONSTANT, BLOCK_TRUNCATED, BLOCK_LOSSLESS = 0, 1, 2
+OP_SUM, OP_MAX, OP_MIN = 0, 1, 2
 
 _lib = None
 
@@ -35,6 +36,10 @@ def lib():
         L.ccz_reduce_step.argtypes = [vp, sz, vp, sz, f32, u32, vp, sz, vp, vp]
         L.ccz_allreduce_sim.restype = i32
         L.ccz_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp]
+        L.ccz_reduce_step_op.restype = i32
+        L.ccz_reduce_step_op.argtypes = [vp, sz, vp, sz, f32, u32, i32, vp, sz, vp, vp]
+        L.ccz_allreduce_sim_op.restype = i32
+        L.ccz_allreduce_sim_op.argtypes = [vp, vp, i32, sz, f32, u32, i32, vp]
         L.ccz_bcast_sim.restype = i32
         L.ccz_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp]
         _lib = L
@@ -95,25 +100,25 @@ def decompress(stream, n, block_len=128, sequential=False):
     return out
 
 
-def reduce_step(stream, local, eb, block_len=128, want_sum=False):
+def reduce_step(stream, local, eb, block_len=128, want_sum=False, op=OP_SUM):
     stream = np.ascontiguousarray(stream, dtype=np.uint8)
     local = _f32(local)
     cap = compress_bound(local.size, block_len)
     out = np.zeros(cap, dtype=np.uint8)
     nbytes = ctypes.c_uint64(0)
     s = np.empty_like(local) if want_sum else None
-    _check(lib().ccz_reduce_step(_ptr(stream), stream.size, _ptr(local), local.size, eb, block_len, _ptr(out), cap,
-                                 ctypes.byref(nbytes), _ptr(s) if want_sum else None))
+    _check(lib().ccz_reduce_step_op(_ptr(stream), stream.size, _ptr(local), local.size, eb, block_len, op, _ptr(out),
+                                    cap, ctypes.byref(nbytes), _ptr(s) if want_sum else None))
     return (out[: nbytes.value].copy(), s) if want_sum else out[: nbytes.value].copy()
 
 
-def allreduce_sim(x, eb, block_len=128):
+def allreduce_sim(x, eb, block_len=128, op=OP_SUM):
     """x: [P, n] fp32.  Returns (out [P, n], bytes_moved)."""
     x = _f32(x)
     P, n = x.shape
     out = np.empty_like(x)
     moved = ctypes.c_uint64(0)
-    _check(lib().ccz_allreduce_sim(_ptr(x), _ptr(out), P, n, eb, block_len, ctypes.byref(moved)))
+    _check(lib().ccz_allreduce_sim_op(_ptr(x), _ptr(out), P, n, eb, block_len, op, ctypes.byref(moved)))
     return out, moved.value
 
 

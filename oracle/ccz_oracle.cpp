@@ -439,15 +439,33 @@ int ccz_decompress_sequential(const uint8_t* in, size_t in_bytes, size_t n, uint
 
 int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L,
                     uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
+  return ccz_reduce_step_op(in, in_bytes, local, n, eb, L, CCZ_OP_SUM, out, cap, out_bytes, sum_out);
+}
+
+/* The reduction of the collective-computation framework is Sum, Max or Min (Sec. III-B).
+ *   SUM: one rounded fp32 add.  IEEE 754 leaves the payload of a NaN result open (and the paper never
+ *        mentions NaN); so that the sum is one well-defined bit pattern on every machine, a NaN sum is
+ *        stored as the quiet NaN 0x7FFFFFFF.
+ *   MAX: a (the decoded value) if a > b or b is a NaN, else b (the local value); a pure selection, so the
+ *        result is one of the two bit patterns.  MIN likewise with <.  (With equal values, e.g. -0 and
+ *        +0, the local value is taken.) */
+int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L, int op,
+                       uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
   if (!local && n) return CCZ_ERR_INVALID_ARG;
+  if (op != CCZ_OP_SUM && op != CCZ_OP_MAX && op != CCZ_OP_MIN) return CCZ_ERR_INVALID_ARG;
   std::vector<float> s(n);
   int rc = ccz_decompress(in, in_bytes, n, L, s.data());
   if (rc != CCZ_OK) return rc;
   for (size_t i = 0; i < n; ++i) {
-    float t = s[i] + local[i];
-    /* IEEE 754 leaves the payload of a NaN result open (and the paper never mentions NaN); so that the
-     * sum is one well-defined bit pattern on every machine, a NaN sum is stored as the quiet NaN 0x7FFFFFFF. */
-    if (t != t) t = float_of(0x7FFFFFFFu);
+    float a = s[i], b = local[i], t;
+    if (op == CCZ_OP_SUM) {
+      t = a + b;
+      if (t != t) t = float_of(0x7FFFFFFFu);
+    } else if (op == CCZ_OP_MAX) {
+      t = (a > b || b != b) ? a : b;
+    } else {
+      t = (a < b || b != b) ? a : b;
+    }
     s[i] = t;
   }
   rc = ccz_compress(s.data(), n, eb, L, out, cap, out_bytes);
@@ -458,7 +476,13 @@ int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size
 }
 
 int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, uint32_t L, uint64_t* bytes_moved) {
+  return ccz_allreduce_sim_op(in, out, P, n, eb, L, CCZ_OP_SUM, bytes_moved);
+}
+
+int ccz_allreduce_sim_op(const float* in, float* out, int P, size_t n, float eb, uint32_t L, int op,
+                         uint64_t* bytes_moved) {
   if (P < 1 || ((!in || !out) && n)) return CCZ_ERR_INVALID_ARG;
+  if (op != CCZ_OP_SUM && op != CCZ_OP_MAX && op != CCZ_OP_MIN) return CCZ_ERR_INVALID_ARG;
   if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
   size_t C = ccz_chunk_len(n, P, L);
   uint64_t moved = 0;
@@ -487,8 +511,8 @@ int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, ui
       int r = (c + k) % P;
       uint64_t nbytes = 0;
       float* sum_out = (k == P - 1) ? out + (size_t)owner * n + lo : nullptr;
-      rc = ccz_reduce_step(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, sb.data(), cap, &nbytes,
-                           sum_out);
+      rc = ccz_reduce_step_op(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, op, sb.data(), cap,
+                              &nbytes, sum_out);
       if (rc != CCZ_OK) return rc;
       sa.swap(sb);
       bytes = nbytes;

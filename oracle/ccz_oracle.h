@@ -47,6 +47,7 @@ enum {
 };
 
 enum { CCZ_BLOCK_CONSTANT = 0, CCZ_BLOCK_TRUNCATED = 1, CCZ_BLOCK_LOSSLESS = 2 };
+enum { CCZ_OP_SUM = 0, CCZ_OP_MAX = 1, CCZ_OP_MIN = 2 }; /* reductions analysed in Sec. III-B */
 
 /* Worst-case stream size for n values in blocks of block_len. */
 size_t ccz_compress_bound(size_t n, uint32_t block_len);
@@ -77,10 +78,17 @@ int ccz_decompress_sequential(const uint8_t* in, size_t in_bytes, size_t n, uint
 int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb,
                     uint32_t block_len, uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out);
 
+/* The same round with the reduction chosen: op = CCZ_OP_SUM / MAX / MIN (Sec. III-B, Theorems 1 and 2). */
+int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb,
+                       uint32_t block_len, int op, uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out);
+
 /* C-Allreduce (Sec. III-E) replayed over P virtual ranks: in and out are [P][n], rank-major.
  * bytes_moved (nullable) = total compressed bytes that would cross the network. */
 int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, uint32_t block_len,
                       uint64_t* bytes_moved);
+
+int ccz_allreduce_sim_op(const float* in, float* out, int P, size_t n, float eb, uint32_t block_len, int op,
+                         uint64_t* bytes_moved);
 
 /* C-Bcast (mode 0) / C-Scatter (mode 1) over P virtual ranks, root = rank 0.
  * out_rank_stride is in floats; rank i's output starts at out + i*out_rank_stride.

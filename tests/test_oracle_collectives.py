@@ -130,3 +130,51 @@ def test_chunk_rule():
     assert ccz.chunk_len(16777216, 8) == 2097152
     assert ccz.chunk_len(1000, 3) == 384
     assert ccz.chunk_len(100, 8) == 128     # later chunks are empty
+
+
+# ---- Max / Min reductions (Sec. III-B, Theorem 2) -----------------------------------------------------------
+
+@pytest.mark.parametrize("op", [ccz.OP_MAX, ccz.OP_MIN])
+def test_max_min_reduce_step_is_a_selection(op):
+    x, eb = ranks_c3(2)
+    a, b = x[0], x[1].copy()
+    b[7] = np.nan                          # a NaN local value loses against the decoded one
+    s0 = ccz.compress(a, eb)
+    ahat = ccz.decompress(s0, a.size)
+    s1, total = ccz.reduce_step(s0, b, eb, want_sum=True, op=op)
+    pick = np.fmax if op == ccz.OP_MAX else np.fmin      # textbook max / min that ignores NaN
+    assert np.array_equal(total, pick(ahat, b))
+    # the result is one of the two inputs, bit for bit
+    tb, ab, bb = total.view(np.uint32), ahat.view(np.uint32), b.view(np.uint32)
+    assert np.all((tb == ab) | (tb == bb))
+    d = ccz.decompress(s1, a.size)
+    assert np.abs(d.astype(np.float64) - total.astype(np.float64)).max() <= float(eb)
+
+
+@pytest.mark.parametrize("op", [ccz.OP_MAX, ccz.OP_MIN])
+@pytest.mark.parametrize("P,n", [(2, 5000), (4, 128 * 37 + 4), (8, 24 * 24 * 32)])
+def test_max_min_allreduce_within_P_eb(op, P, n):
+    x, eb = ranks_c3(P)
+    x = np.ascontiguousarray(x[:, :n])
+    out, moved = ccz.allreduce_sim(x, eb, op=op)
+    exact = x.max(axis=0) if op == ccz.OP_MAX else x.min(axis=0)
+    err = np.abs(out.astype(np.float64) - exact[None, :].astype(np.float64))
+    # every round perturbs the running extreme by at most eb, and max/min are 1-Lipschitz
+    assert err.max() <= P * float(eb)
+    # a selection never adds rounding: with all-constant identical blocks the extreme is exact
+    y = np.full((P, 4096), 0.375, dtype=np.float32)
+    out2, _ = ccz.allreduce_sim(y, eb, op=op)
+    assert np.all(out2 == np.float32(0.375))
+    # soft check (Theorem 2): the error variance stays below 2 sigma^2 with sigma = eb/3
+    assert err.std() <= np.sqrt(2.0) * float(eb)
+
+
+def test_max_min_equal_values_take_the_local_one():
+    a = np.zeros(128, dtype=np.float32)               # decoded side: +0
+    b = np.full(128, -0.0, dtype=np.float32)          # local side: -0
+    s0 = ccz.compress(a, np.float32(1e-3))
+    for op in (ccz.OP_MAX, ccz.OP_MIN):
+        _, total = ccz.reduce_step(s0, b, np.float32(1e-3), want_sum=True, op=op)
+        assert total.tobytes() == b.tobytes()
+    with pytest.raises(ccz.OracleError):
+        ccz.reduce_step(s0, b, np.float32(1e-3), op=7)
