@@ -62,6 +62,7 @@ typedef enum {
 #define CCOLL_MAX_VALUES ((size_t)1 << 29) /* values per stream (2 GiB of fp32) */
 
 enum { CCOLL_BCAST = 0, CCOLL_SCATTER = 1 };
+enum { CCOLL_SUM = 0, CCOLL_MAX = 1, CCOLL_MIN = 2 }; /* reductions of the computation framework, Sec. III-B */
 
 /* Worst-case stream size in bytes for n values (0 if block_len is unsupported).  Output buffers of
  * ccoll_compress / ccoll_reduce_step must hold this many bytes. */
@@ -110,6 +111,13 @@ int ccoll_decompress(const void* in, size_t in_bytes, size_t n, uint32_t block_l
 int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
                       uint32_t block_len, void* out, uint64_t* out_bytes, float* sum_out, void* stream);
 
+/* The same round with the reduction chosen (Sec. III-B analyses Sum, Max and Min; Theorems 1 and 2).
+ *   op  CCOLL_SUM: as ccoll_reduce_step.  CCOLL_MAX / CCOLL_MIN: the decoded value if it is greater / smaller
+ *       than the local one or the local one is a NaN, else the local value — a selection, never rounded.
+ * `sum_out`, if given, receives the uncompressed reduced values.  Any other op: CCOLL_ERR_INVALID_ARG. */
+int ccoll_reduce_step_op(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
+                         uint32_t block_len, int op, void* out, uint64_t* out_bytes, float* sum_out, void* stream);
+
 /* C-Allreduce (SUM) replayed over P virtual ranks in one GPU (Sec. III-E; reduce-scatter per Fig. 4, then
  * the compress-once allgather of Sec. III-E-1).
  *   in   [P][n] fp32 rank-major;  out  [P][n] fp32 rank-major (must not alias in)
@@ -121,6 +129,10 @@ int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_
  * Launches: 1 batched compress, P-1 batched fused reduce steps, 1 batched decode.  P = 1 copies in to out. */
 int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
                         uint64_t* bytes_moved, void* stream);
+
+/* ccoll_allreduce_sim with the reduction chosen (CCOLL_SUM / CCOLL_MAX / CCOLL_MIN, as ccoll_reduce_step_op). */
+int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                           int op, uint64_t* bytes_moved, void* stream);
 
 /* C-Bcast / C-Scatter replayed over P virtual ranks, root = rank 0 (Sec. III-A-1: the root compresses each
  * chunk once, the tree forwards compressed bytes, every receiver decompresses once).

@@ -12,12 +12,13 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CORRUPT, ERR_TIMEOUT, ERR_CUDA = range(7)
 BCAST, SCATTER = 0, 1
+SUM, MAX, MIN = 0, 1, 2
 BLOCK_LEN = 128
 _NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CAPACITY", 4: "CORRUPT", 5: "TIMEOUT", 6: "CUDA"}
 
 EXPORTS = ("ccoll_compress_bound", "ccoll_chunk_len", "ccoll_workspace_bytes", "ccoll_set_workspace",
            "ccoll_get_status", "ccoll_compress", "ccoll_decompress", "ccoll_reduce_step", "ccoll_allreduce_sim",
-           "ccoll_bcast_sim", "ccoll_compress_noalloc")
+           "ccoll_bcast_sim", "ccoll_compress_noalloc", "ccoll_reduce_step_op", "ccoll_allreduce_sim_op")
 
 _lib = None
 
@@ -55,6 +56,10 @@ def lib():
     L.ccoll_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp, vp]
     L.ccoll_bcast_sim.restype = i32
     L.ccoll_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp, vp]
+    L.ccoll_reduce_step_op.restype = i32
+    L.ccoll_reduce_step_op.argtypes = [vp, sz, vp, sz, f32, u32, i32, vp, vp, vp, vp]
+    L.ccoll_allreduce_sim_op.restype = i32
+    L.ccoll_allreduce_sim_op.argtypes = [vp, vp, i32, sz, f32, u32, i32, vp, vp]
     L.ccoll_compress_noalloc.restype = i32
     L.ccoll_compress_noalloc.argtypes = [vp, sz, f32, u32, vp, vp, vp, vp]
     _lib = L
@@ -136,6 +141,19 @@ def ccoll_reduce_step(in_buf, in_bytes, local, eb, out, out_bytes=None, sum_out=
                                    _ptr(out_bytes), _ptr(sum_out), _stream(stream)), "ccoll_reduce_step")
 
 
+def ccoll_reduce_step_op(in_buf, in_bytes, local, eb, op, out, out_bytes=None, sum_out=None, block_len=BLOCK_LEN,
+                         stream=None):
+    _check(lib().ccoll_reduce_step_op(_ptr(in_buf), in_bytes, _ptr(local), local.numel(), eb, block_len, op,
+                                      _ptr(out), _ptr(out_bytes), _ptr(sum_out), _stream(stream)),
+           "ccoll_reduce_step_op")
+
+
+def ccoll_allreduce_sim_op(x, out, eb, op, bytes_moved=None, block_len=BLOCK_LEN, stream=None):
+    P, n = x.shape
+    _check(lib().ccoll_allreduce_sim_op(_ptr(x), _ptr(out), P, n, eb, block_len, op, _ptr(bytes_moved),
+                                        _stream(stream)), "ccoll_allreduce_sim_op")
+
+
 def ccoll_allreduce_sim(x, out, eb, bytes_moved=None, block_len=BLOCK_LEN, stream=None):
     P, n = x.shape
     _check(lib().ccoll_allreduce_sim(_ptr(x), _ptr(out), P, n, eb, block_len, _ptr(bytes_moved), _stream(stream)),
@@ -175,24 +193,24 @@ def decompress(stream_buf, n, block_len=BLOCK_LEN):
     return out
 
 
-def reduce_step(stream_buf, local, eb, want_sum=False, block_len=BLOCK_LEN):
+def reduce_step(stream_buf, local, eb, want_sum=False, block_len=BLOCK_LEN, op=SUM):
     n = local.numel()
     ensure_workspace(n)
     out = torch.empty(ccoll_compress_bound(n, block_len), dtype=torch.uint8, device=local.device)
     nbytes = torch.zeros(1, dtype=torch.int64, device=local.device)
     s = torch.empty_like(local) if want_sum else None
-    ccoll_reduce_step(stream_buf, stream_buf.numel(), local, eb, out, nbytes, s, block_len)
+    ccoll_reduce_step_op(stream_buf, stream_buf.numel(), local, eb, op, out, nbytes, s, block_len)
     _check(ccoll_get_status(), "ccoll_reduce_step (device)")
     out = out[: int(nbytes.item())]
     return (out, s) if want_sum else out
 
 
-def allreduce_sim(x, eb, block_len=BLOCK_LEN):
+def allreduce_sim(x, eb, block_len=BLOCK_LEN, op=SUM):
     P, n = x.shape
     ensure_workspace(n, P)
     out = torch.empty_like(x)
     moved = torch.zeros(1, dtype=torch.int64, device=x.device)
-    ccoll_allreduce_sim(x, out, eb, moved, block_len)
+    ccoll_allreduce_sim_op(x, out, eb, op, moved, block_len)
     _check(ccoll_get_status(), "ccoll_allreduce_sim (device)")
     return out, int(moved.item())
 

@@ -186,8 +186,15 @@ int ccoll_decompress(const void* in, size_t in_bytes, size_t n, uint32_t block_l
 
 int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
                       uint32_t block_len, void* out, uint64_t* out_bytes, float* sum_out, void* stream) {
+  return ccoll_reduce_step_op(in, in_bytes, local, n, abs_err_bound, block_len, CCOLL_SUM, out, out_bytes, sum_out,
+                              stream);
+}
+
+int ccoll_reduce_step_op(const void* in, size_t in_bytes, const float* local, size_t n, float abs_err_bound,
+                         uint32_t block_len, int op, void* out, uint64_t* out_bytes, float* sum_out, void* stream) {
   int rc = check_common(n, abs_err_bound, block_len);
   if (rc != CCOLL_OK) return rc;
+  if (op != CCOLL_SUM && op != CCOLL_MAX && op != CCOLL_MIN) return CCOLL_ERR_INVALID_ARG;
   if (!in || !out || (!local && n) || !aligned16(in) || !aligned16(out) || !aligned16(local) || !aligned16(sum_out) ||
       (reinterpret_cast<uintptr_t>(out_bytes) & 7u) || in == out || in == (const void*)local)
     return CCOLL_ERR_INVALID_ARG;
@@ -206,6 +213,7 @@ int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_
   b.out_cap = ccoll_compress_bound(n, block_len);
   b.out_bytes = out_bytes;
   b.sum_out = sum_out;
+  b.op = op;
   size_t G = groups_of(n);
   b.tiles_per_job = (uint32_t)G;
   b.state_stride = (uint32_t)(G + (G + 31) / 32);
@@ -215,7 +223,13 @@ int ccoll_reduce_step(const void* in, size_t in_bytes, const float* local, size_
 
 int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
                         uint64_t* bytes_moved, void* stream) {
+  return ccoll_allreduce_sim_op(in, out, P, n, abs_err_bound, block_len, CCOLL_SUM, bytes_moved, stream);
+}
+
+int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                           int op, uint64_t* bytes_moved, void* stream) {
   if (P < 1 || (size_t)P > kMaxJobs) return CCOLL_ERR_INVALID_ARG;
+  if (op != CCOLL_SUM && op != CCOLL_MAX && op != CCOLL_MIN) return CCOLL_ERR_INVALID_ARG;
   size_t C = ccoll_chunk_len(n, P, block_len);
   int rc = check_common(C, abs_err_bound, block_len);
   if (rc != CCOLL_OK) return rc;
@@ -248,6 +262,7 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
     b.n = n;
     b.P = P;
     b.rot = k;  // in round k, chunk c is at rank (c + k) mod P
+    b.op = op;
     b.s_stride = S;
     b.out_cap = S;
     b.moved = bytes_moved;

@@ -730,15 +730,24 @@ __device__ __noinline__ float4 decode_quad_generic(const uint32_t* img, DecodeCu
                      __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
 }
 
+// One reduction of the collective-computation framework (Sec. III-B): a = decoded value, b = local value.
+// Sum: one rounded add (a NaN result is the GPU's canonical 0x7FFFFFFF).  Max / Min: a pure selection, a if
+// it beats b or b is a NaN, else b.
+__device__ __forceinline__ float reduce_op(float a, float b, int op) {
+  if (op == 0) return __fadd_rn(a, b);
+  if (op == 1) return (a > b || b != b) ? a : b;
+  return (a < b || b != b) ? a : b;
+}
+
 // Decode the lane's 32 values of group g into v[].  Returns false (for the whole CTA) on a corrupt group.
 // The group's payload must already be staged in sm.img (and visible).  nblk = blocks in the group.
 // kToSlice = false: the values are returned in v[] (fully unrolled loops).  kToSlice = true (fused reduce):
-// each decoded quad is ADDED to the quad of local values waiting in the lane's slice and the sum is written
+// each decoded quad is REDUCED (op) with the quad of local values waiting in the lane's slice and the result is written
 // back there; the loops are then unrolled only twice, which keeps the fused kernel inside the instruction
 // cache.
 template <bool kToSlice>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8], float4* slice4) {
+                                             float4 (&v)[8], float4* slice4, int op = 0) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
@@ -853,7 +862,8 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   auto put = [&](int j, const float4& r) {
     if (kToSlice) {
       const float4 a = slice4[j];
-      slice4[j] = make_float4(__fadd_rn(r.x, a.x), __fadd_rn(r.y, a.y), __fadd_rn(r.z, a.z), __fadd_rn(r.w, a.w));
+      slice4[j] = make_float4(reduce_op(r.x, a.x, op), reduce_op(r.y, a.y, op), reduce_op(r.z, a.z, op),
+                              reduce_op(r.w, a.w, op));
     } else {
       v[j] = r;
     }
@@ -1013,7 +1023,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     __syncthreads();  // the image and the local values in the rows are complete
     TL(1);
     // decoded + local, one rounded add per value, left in the lane's slice
-    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice);
+    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice, b.op);
   }
   TL(2);
   if (!ok) {

@@ -261,3 +261,28 @@ def test_many_virtual_ranks():
     with pytest.raises(B.CcollError) as e:
         B.ccoll_bcast_sim(dev(root), torch.empty(8, device="cuda"), 0, 1025, eb)
     assert e.value.code == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("op", [B.MAX, B.MIN])
+def test_max_min_reduce_step_and_allreduce_match_oracle(op):
+    c = fields.config3(P=4, shape=(32, 32, 40), sigma=3.0)
+    x, eb = c["x"].numpy().copy(), float(np.float32(c["eb"]))
+    x[1, 7] = np.nan                 # a NaN on the local side never wins
+    x[0, 300] = np.inf
+    x[1, 900:1028] = -0.0            # equal values (+-0): the local one is taken
+    x[0, 900:1028] = 0.0
+    for n in (x.shape[1], 4096 + 130, 5):
+        a, b_ = x[0, :n], x[1, :n]
+        s0 = ccz.compress(a, eb)
+        ref, rtot = ccz.reduce_step(s0, b_, eb, want_sum=True, op=op)
+        got, gtot = B.reduce_step(dev(s0), dev(b_), eb, want_sum=True, op=op)
+        assert np.array_equal(got.cpu().numpy(), ref)
+        assert gtot.cpu().numpy().tobytes() == rtot.tobytes()
+    n = 128 * 37 + 4
+    xs = np.ascontiguousarray(x[:, :n])
+    ref, ref_moved = ccz.allreduce_sim(xs, eb, op=op)
+    got, moved = B.allreduce_sim(dev(xs), eb, op=op)
+    assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
+    with pytest.raises(B.CcollError) as e:
+        B.reduce_step(dev(s0), dev(b_), eb, op=5)
+    assert e.value.code == B.ERR_INVALID_ARG
