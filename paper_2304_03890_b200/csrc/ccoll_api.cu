@@ -159,7 +159,7 @@ int ccoll_compress(const float* in, size_t n, float abs_err_bound, uint32_t bloc
   b.out_bytes = out_bytes;
   size_t G = groups_of(n);
   b.tiles_per_job = (uint32_t)G;
-  b.state_stride = (uint32_t)(G + (G + 31) / 32);
+  b.state_stride = state_words((uint32_t)G);
   if (!launch_compress(b, (uint32_t)(G ? G : 1), 1, s)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
@@ -216,7 +216,7 @@ int ccoll_reduce_step_op(const void* in, size_t in_bytes, const float* local, si
   b.op = op;
   size_t G = groups_of(n);
   b.tiles_per_job = (uint32_t)G;
-  b.state_stride = (uint32_t)(G + (G + 31) / 32);
+  b.state_stride = state_words((uint32_t)G);
   if (!launch_reduce(b, (uint32_t)(G ? G : 1), 1, s)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
@@ -268,7 +268,7 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
     b.moved = bytes_moved;
     b.moved_mult = (k == P - 1) ? (uint32_t)(P - 1) : 1u;
     b.tiles_per_job = (uint32_t)Gc;
-    b.state_stride = (uint32_t)(Gc + (Gc + 31) / 32);
+    b.state_stride = state_words((uint32_t)Gc);
     if (k == 0) {
       b.sout = buf[cur];
       b.out_bytes = bytes[cur];
@@ -334,7 +334,7 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   b.out_cap = S;
   b.out_bytes = bytes;
   b.tiles_per_job = (uint32_t)Gc;
-  b.state_stride = (uint32_t)(Gc + (Gc + 31) / 32);
+  b.state_stride = state_words((uint32_t)Gc);
   if (!launch_compress(b, (uint32_t)(Gc ? Gc : 1), (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   if ((rc = check_launch()) != CCOLL_OK) return rc;
   if (chunk_bytes &&

@@ -32,7 +32,6 @@ __device__ unsigned long long g_timeline[8192 * 16];
 #define TL(slot) do {} while (0)
 #endif
 namespace {
-
 constexpr uint32_t kFull = 0xffffffffu;
 constexpr int kSliceVals = 32;                      // values per lane
 constexpr int kSliceBytes = 144;                    // 128 data bytes + 16 pad
@@ -105,21 +104,22 @@ __device__ __forceinline__ void or_u64(uint32_t* img, uint32_t off, uint32_t lo,
 // geometry
 // ---------------------------------------------------------------------------------------------------
 struct JobGeom {
-  uint64_t lo;      // first value of the job inside the rank buffer
-  uint64_t len;     // values in the job
+  uint32_t lo;      // first value of the job inside the rank buffer
+  uint32_t len;     // values in the job
   uint32_t nb;      // blocks
   uint32_t G;       // groups
   uint32_t m_last;  // values in the job's last block (1..128; 0 if the job is empty)
 };
-__device__ __forceinline__ JobGeom job_geom(uint64_t n, uint64_t C, uint32_t y) {
+// A rank buffer holds at most 2^29 values (the entry points check it), so value indices fit 32 bits.
+__device__ __forceinline__ JobGeom job_geom(uint64_t n64, uint64_t C64, uint32_t y) {
   JobGeom j;
-  uint64_t lo = (uint64_t)y * C, hi = lo + C;
-  j.lo = lo < n ? lo : n;
-  hi = hi < n ? hi : n;
-  j.len = hi - j.lo;
-  j.nb = (uint32_t)((j.len + kL - 1) / kL);
+  const uint32_t n = (uint32_t)n64, C = (uint32_t)C64;
+  const uint64_t lo64 = (uint64_t)y * C;
+  j.lo = lo64 < n ? (uint32_t)lo64 : n;
+  j.len = min(C, n - j.lo);
+  j.nb = (j.len + kL - 1) / kL;
   j.G = (j.nb + kGroupBlocks - 1) / kGroupBlocks;
-  j.m_last = (uint32_t)(j.len - (uint64_t)(j.nb ? j.nb - 1 : 0) * kL);
+  j.m_last = j.len - (j.nb ? j.nb - 1 : 0) * kL;
   return j;
 }
 // What a thread owns in group g: its block's value count and its own valid values.
@@ -128,8 +128,6 @@ struct LaneGeom {
   uint32_t t;      // slice inside the block (tid % 4)
   uint32_t m_blk;  // values in the block (0 = the block does not exist)
   uint32_t nv;     // valid values in this lane's slice (0..32)
-  uint32_t nfull;  // complete slices in the whole group
-  uint64_t first;  // index (inside the job) of the slice's first value
 };
 __device__ __forceinline__ LaneGeom lane_geom(const JobGeom& jg, uint32_t g) {
   LaneGeom lg;
@@ -140,10 +138,11 @@ __device__ __forceinline__ LaneGeom lane_geom(const JobGeom& jg, uint32_t g) {
   lg.m_blk = gblk < jg.nb ? (gblk == jg.nb - 1 ? jg.m_last : (uint32_t)kL) : 0u;
   int nv = (int)lg.m_blk - (int)(kSliceVals * lg.t);
   lg.nv = (uint32_t)(nv < 0 ? 0 : (nv > kSliceVals ? kSliceVals : nv));
-  uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
-  lg.nfull = (uint32_t)((rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues) / kSliceVals);
-  lg.first = (uint64_t)gblk * kL + (uint64_t)kSliceVals * lg.t;
   return lg;
+}
+// values of group g that exist (4096 except in the job's last group)
+__device__ __forceinline__ uint32_t group_count(const JobGeom& jg, uint32_t g) {
+  return min((uint32_t)kGroupValues, jg.len - g * (uint32_t)kGroupValues);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -176,32 +175,52 @@ __device__ __forceinline__ void zero_image(uint32_t* img) {  // a barrier must f
 // the CTA that currently occupies the SM slot that later CTA will get, so its loads find the data in L2.
 __device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg, uint32_t g) {
   if (g >= jg.G) return;
-  const uint64_t first = (uint64_t)g * kGroupValues + 32u * threadIdx.x;
+  const uint32_t first = g * (uint32_t)kGroupValues + 32u * threadIdx.x;
   if (first < jg.len) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + first));
 }
+// Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
+// (128-bit streaming loads) and scatters them into the padded slices; in round r thread tid moves the
+// float4 number r*128 + tid of the group.  A __syncthreads must follow before the slices are read.
+// (Letting every lane fetch its own 128 bytes with 256-bit loads needs no transposition and no barrier, but
+// each such load touches 32 lines and the load/store pipe, already the busiest unit here, made it slower.)
 __device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
-  const uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
-  const uint32_t cnt = (uint32_t)(rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues);
-  const float* src = x + (uint64_t)g * kGroupValues;
-  float4 t[8];
+  const uint32_t cnt = group_count(jg, g);
+  const float* src = x + (size_t)g * kGroupValues;
+  float4* dst = reinterpret_cast<float4*>(rows + (tid >> 3) * kSliceBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kSliceBytes / 16;  // float4s between a thread's rounds
+  if (cnt == (uint32_t)kGroupValues) {  // a complete group: no bounds to watch
+    float4 t[8];
 #pragma unroll
+    for (int r = 0; r < 8; ++r) t[r] = __ldcs(reinterpret_cast<const float4*>(src) + r * kThreads + tid);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) dst[r * kRoundStride] = t[r];
+    return;
+  }
+#pragma unroll 1
   for (int r = 0; r < 8; ++r) {
     const uint32_t f = (uint32_t)r * kThreads + tid;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (4u * f + 4u <= cnt) {
-      t[r] = __ldcs(reinterpret_cast<const float4*>(src) + f);
+      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
     } else {
-      t[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (4u * f + 0u < cnt) t[r].x = __ldcs(src + 4u * f + 0u);
-      if (4u * f + 1u < cnt) t[r].y = __ldcs(src + 4u * f + 1u);
-      if (4u * f + 2u < cnt) t[r].z = __ldcs(src + 4u * f + 2u);
+      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
     }
+    dst[r * kRoundStride] = v;
   }
-#pragma unroll
-  for (int r = 0; r < 8; ++r) {
-    const uint32_t f = (uint32_t)r * kThreads + tid;
-    *reinterpret_cast<float4*>(rows + (f >> 3) * kSliceBytes + 16u * (f & 7u)) = t[r];
+}
+// Ragged slices: values past the end of the data are replaced by the block's first value, so that they
+// cannot change min or max.  (The first value of block b is the first value of slice 4b.)  Whole warp.
+__device__ __forceinline__ void pad_ragged(uint8_t* rows, const LaneGeom& lg) {
+  __syncwarp();
+  if (lg.nv < (uint32_t)kSliceVals) {
+    const float f = *reinterpret_cast<const float*>(rows + (threadIdx.x & ~3u) * kSliceBytes);
+    float* x = reinterpret_cast<float*>(rows + threadIdx.x * kSliceBytes);
+    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) x[i] = f;
   }
+  __syncwarp();
 }
 // Put the lane's 32 values (held in v) into its slice of the rows.
 __device__ __forceinline__ void write_slice(uint8_t* rows, const float4 (&v)[8]) {
@@ -213,13 +232,19 @@ __device__ __forceinline__ void write_slice(uint8_t* rows, const float4 (&v)[8])
 // mirror image of load_rows).  A __syncthreads must separate it from the writes of the slices.
 __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
-  const uint64_t rest = jg.len - (uint64_t)g * kGroupValues;
-  const uint32_t cnt = (uint32_t)(rest < (uint64_t)kGroupValues ? rest : (uint64_t)kGroupValues);
-  float* dst = out + (uint64_t)g * kGroupValues;
+  const uint32_t cnt = group_count(jg, g);
+  float* dst = out + (size_t)g * kGroupValues;
+  const float4* src = reinterpret_cast<const float4*>(rows + (tid >> 3) * kSliceBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kSliceBytes / 16;
+  if (cnt == (uint32_t)kGroupValues) {
 #pragma unroll
+    for (int r = 0; r < 8; ++r) __stcs(reinterpret_cast<float4*>(dst) + r * kThreads + tid, src[r * kRoundStride]);
+    return;
+  }
+#pragma unroll 1
   for (int r = 0; r < 8; ++r) {
     const uint32_t f = (uint32_t)r * kThreads + tid;
-    const float4 t = *reinterpret_cast<const float4*>(rows + (f >> 3) * kSliceBytes + 16u * (f & 7u));
+    const float4 t = src[r * kRoundStride];
     if (4u * f + 4u <= cnt) {
       __stcs(reinterpret_cast<float4*>(dst) + f, t);
     } else {
@@ -243,18 +268,20 @@ struct Plan {
   bool lossless;
 };
 
-// The loops over a lane's eight quads read the values from the lane's slice and are only unrolled twice:
-// fully unrolled on register arrays the fused kernel outgrew the 32 KB instruction cache (84 % hit rate).
-__device__ __forceinline__ Plan plan_block(const float4* x4, const LaneGeom& lg, float eb, int eb_exp) {
+// Largest and smallest of the lane's 32 values (a NaN wins both), read from the lane's slice.  The loop is
+// unrolled only twice: fully unrolled on register arrays the fused kernel outgrew the 32 KB instruction cache.
+__device__ __forceinline__ void lane_minmax(const float4* x4, float& mx, float& mn) {
   float4 q = x4[0];
-  float mx = max3_nan(max_nan(q.x, q.y), q.z, q.w);
-  float mn = min3_nan(min_nan(q.x, q.y), q.z, q.w);
+  mx = max3_nan(max_nan(q.x, q.y), q.z, q.w);
+  mn = min3_nan(min_nan(q.x, q.y), q.z, q.w);
 #pragma unroll 2
   for (int j = 1; j < 8; ++j) {
     q = x4[j];
     mx = max3_nan(max3_nan(mx, q.x, q.y), q.z, q.w);
     mn = min3_nan(min3_nan(mn, q.x, q.y), q.z, q.w);
   }
+}
+__device__ __forceinline__ Plan plan_block(float mx, float mn, const LaneGeom& lg, float eb, int eb_exp) {
   mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 1));
   mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 1));
   mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 2));
@@ -344,18 +371,33 @@ __device__ __forceinline__ void finish_stage(Stage& st) {
   st.wp[1] = 0u;        // and a zero word behind it for the realigning copy
 }
 
-// Fast path: all 32 values valid, block not lossless.  Values are read from the slice quad by quad; the
-// staged bytes overwrite the slice in place, which is safe because quad j is read before anything is
-// written at or behind its position.
+// Fast path: all 32 values valid, block not lossless.  The lane's byte string is built in a 64-bit big-endian
+// accumulator (hi:lo, its low `pend` bits waiting to be written): a value's stored bytes are its low
+// n = 8 * (stored bytes) bits, appended with two funnel shifts; whenever 32 bits are complete they leave as
+// one word (byte-reversed, since the first byte of the stream is the most significant one).  n comes
+// straight from the leading-zero count of (code xor predecessor); `fix` forces at least one stored byte when
+// the field is 4 bytes wide (lead is capped at 3).  Values are read from the slice quad by quad and the
+// staged words overwrite the slice in place, which is safe because at most 16 bytes are staged per quad and
+// quad j is read before anything is written at or behind its position.
 __device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const Plan& p, uint32_t prev, uint32_t& T_out,
                                                uint32_t& code_lo, uint32_t& code_hi) {
   const uint32_t fix = (p.B == 4u) ? 1u : 0u;
-  const uint32_t cadj = (4u - p.B) * 85u;
+  const uint32_t cadj = (4u - p.B) * (85u << 24);
   const float mu = p.mu;
   const uint32_t sh = p.sh;
-  Stage st = {slice, 0u, 0u, 0u};
-  uint64_t codes = 0ull;
+  uint32_t lo = 0u, hi = 0u, Tb = 0u;  // Tb = bits appended so far; the low (Tb & 31) bits of hi:lo are waiting
+  uint32_t clo = 0u, chi = 0u;
   const float4* x4 = reinterpret_cast<const float4*>(slice);
+  auto put = [&](uint32_t q, uint32_t sa) {
+    const uint32_t n = 32u - sa;
+    const uint32_t t = __funnelshift_lc(0u, q, sa);  // the stored bits, at the top of the word
+    const uint32_t Tn = Tb + n;                      // the only loop-carried add: everything else hangs off it
+    hi = __funnelshift_lc(lo, hi, n);
+    lo = __funnelshift_lc(t, lo, n);
+    if ((Tn ^ Tb) & 32u)  // a word boundary was crossed (n <= 32: at most one)
+      slice[(Tn >> 5) - 1u] = __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123);
+    Tb = Tn;
+  };
 #pragma unroll 2
   for (int j = 0; j < 8; ++j) {
     const float4 x = x4[j];
@@ -364,15 +406,23 @@ __device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const Plan& p, u
     const uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
                    sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
     prev = q3;
-    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field
-    const uint32_t cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) >> 3) - cadj;
-    codes |= (uint64_t)cb << (8 * j);
-    append_quad(st, q0, q1, q2, q3, sa0, sa1, sa2, sa3);
+    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field; the
+    // quad's four codes enter the 64-bit code string from the top, so that after eight quads quad 0 is lowest
+    const uint32_t cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) << 21) - cadj;
+    clo = __funnelshift_r(clo, chi, 8u);
+    chi = (chi >> 8) | cb;
+    put(q0, sa0);
+    put(q1, sa1);
+    put(q2, sa2);
+    put(q3, sa3);
   }
-  finish_stage(st);
-  T_out = st.Tb >> 3;
-  code_lo = (uint32_t)codes;
-  code_hi = (uint32_t)(codes >> 32);
+  const uint32_t pend = Tb & 31u;
+  uint32_t* wp = slice + (Tb >> 5);
+  wp[0] = pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u;  // the last partial word, zero padded
+  wp[1] = 0u;                                                        // and a zero word for the realigning copy
+  T_out = Tb >> 3;
+  code_lo = clo;
+  code_hi = chi;
 }
 
 // General path (ragged slices, lossless blocks): rolled loop over the quads, values re-read from the slice.
@@ -461,6 +511,7 @@ __device__ __forceinline__ uint32_t quad_scan(uint32_t v, uint32_t t, uint32_t l
 // nothing ever waits on a prefix: A[t] = size of tile t; SA[s] = size of super-tile s (32 tiles), written
 // by the super-tile's last tile from the A's it has to read anyway.  Tile g needs A[32s .. g-1] and
 // SA[0 .. s-1]: independent loads spread over the CTA's threads, one round trip once the data is there.
+// (A third level, sums of 1024 tiles, cuts the loads per tile from G/64 to about 36 and was measured slower.)
 // Words carry the launch's epoch, so stale entries read as "not written yet"; every wait is bounded.
 __device__ __forceinline__ uint32_t poll_size(const uint64_t* p, uint32_t epoch, uint32_t* status, bool& bad) {
   uint32_t spins = 0;
@@ -478,53 +529,64 @@ __device__ __forceinline__ uint32_t poll_size(const uint64_t* p, uint32_t epoch,
     __nanosleep(32);
   }
 }
-// Called by every thread of the CTA after A[g] was published.  Adds the group's exclusive prefix (in words)
-// to sm.prefix and raises sm.fail on a poisoned or timed-out entry; both are read after the next barrier.
-__device__ __forceinline__ void find_prefix(Smem& sm, uint64_t* A, uint64_t* SA, uint32_t g, uint32_t G, uint32_t words,
-                                            uint32_t epoch, uint32_t* status) {
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+// Both halves add to sm.prefix and raise sm.fail on a poisoned or timed-out entry; both words are read after
+// the next barrier.  Called by every thread of the CTA after A[g] was published.
+// Warp 0: the sizes of the earlier tiles of the own super-tile; the super-tile's last tile also publishes
+// SA[s].  That tile calls this BEFORE it places its bytes in the image, every other tile after: the tiles of
+// the next super-tile then find SA[s] one round trip after A[32s+31] instead of one placement and a round
+// trip later.
+struct SizeWords {
+  uint64_t *A, *SA;
+};
+__device__ __forceinline__ SizeWords size_words(const EncodeBatch& b, uint32_t y) {
+  SizeWords w;
+  w.A = b.tile_state + (uint64_t)y * b.state_stride;
+  w.SA = w.A + b.tiles_per_job;
+  return w;
+}
+__device__ __forceinline__ void prefix_own_super_tile(Smem& sm, const SizeWords& w, uint32_t g, uint32_t G,
+                                                      uint32_t words, uint32_t epoch, uint32_t* status) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  if (tid >= 32u) return;
   const uint32_t s = g >> 5, r = g & 31u;
   uint32_t sum = 0u;
   bool bad = false;
-  if (warp == 0) {
-    if (lane < r) sum = poll_size(&A[32u * s + lane], epoch, status, bad);
-    sum = __reduce_add_sync(kFull, sum);
-    bad = __any_sync(kFull, bad);
-    if (lane == 0) {
-      if (r == 31u || g == G - 1u)
-        st_relaxed_u64(&SA[s], pack_state(epoch, bad ? kFlagPoison : kFlagAggregate, sum + words));
-      if (sum) atomicAdd(&sm.prefix, sum);
-      if (bad) atomicOr(&sm.fail, 1u);
-    }
-  } else {
-    for (uint32_t t = tid - 32u; t < s; t += kThreads - 32u) sum += poll_size(&SA[t], epoch, status, bad);
-    sum = __reduce_add_sync(kFull, sum);
-    bad = __any_sync(kFull, bad);
-    if (lane == 0) {
-      if (sum) atomicAdd(&sm.prefix, sum);
-      if (bad) atomicOr(&sm.fail, 1u);
-    }
+  if (lane < r) sum = poll_size(&w.A[32u * s + lane], epoch, status, bad);
+  sum = __reduce_add_sync(kFull, sum);
+  bad = __any_sync(kFull, bad);
+  if (lane == 0) {
+    if (r == 31u || g == G - 1u)
+      st_relaxed_u64(&w.SA[s], pack_state(epoch, bad ? kFlagPoison : kFlagAggregate, sum + words));
+    if (sum) atomicAdd(&sm.prefix, sum);
+    if (bad) atomicOr(&sm.fail, 1u);
+  }
+}
+// Warps 1-3: the earlier super-tiles.
+__device__ __forceinline__ void prefix_earlier_super_tiles(Smem& sm, const SizeWords& w, uint32_t g, uint32_t epoch,
+                                                           uint32_t* status) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  if (tid < 32u) return;
+  const uint32_t s = g >> 5;
+  uint32_t sum = 0u;
+  bool bad = false;
+  for (uint32_t t = tid - 32u; t < s; t += kThreads - 32u) sum += poll_size(&w.SA[t], epoch, status, bad);
+  sum = __reduce_add_sync(kFull, sum);
+  bad = __any_sync(kFull, bad);
+  if (lane == 0) {
+    if (sum) atomicAdd(&sm.prefix, sum);
+    if (bad) atomicOr(&sm.fail, 1u);
   }
 }
 
-// Encode the group whose values the threads hold in v[] (32 per thread), build its payload image, find its
-// place in the stream and copy it out.  The image must have been zeroed (and that made visible by the
-// barrier inside) before the call.
+// Encode the group whose values wait in the lanes' slices (ragged slices already padded; mx, mn = largest and
+// smallest value of the lane's slice): build the payload image, find its place in the stream and copy it
+// out.  The image must have been zeroed (that is made visible by the barrier inside) before the call.
 __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const LaneGeom& lg, const EncodeBatch& b,
-                                             const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout) {
+                                             const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout, float mx,
+                                             float mn, bool tail) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   uint32_t* slice = reinterpret_cast<uint32_t*>(rows + tid * kSliceBytes);
-  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
-
-  if (tail && lg.nv < (uint32_t)kSliceVals) {
-    // Ragged slice (rare): values past the end of the data are replaced by the block's first value, so that
-    // they cannot change min or max.  (The first value of block b is the first value of slice 4b.)
-    const float f = *reinterpret_cast<const float*>(rows + (tid & ~3u) * kSliceBytes);
-    float* x = reinterpret_cast<float*>(slice);
-    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) x[i] = f;
-  }
-  if (tail) __syncwarp();
-  Plan p = plan_block(reinterpret_cast<const float4*>(slice), lg, b.eb, b.eb_exp);
+  Plan p = plan_block(mx, mn, lg, b.eb, b.eb_exp);
   // code of the value just before this lane's first one (0 at the start of a block)
   uint32_t prev = __shfl_up_sync(kFull, code_of(reinterpret_cast<const float*>(slice)[kSliceVals - 1], p), 1);
   if (lg.t == 0u) prev = 0u;
@@ -556,15 +618,16 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const Lane
   const uint32_t words = (raw + 3u) >> 2;
   const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
 
-  uint64_t* A = b.tile_state + (uint64_t)y * b.state_stride;
-  uint64_t* SA = A + b.tiles_per_job;
+  const SizeWords sw = size_words(b, y);
   if (warp == 0) {
-    if (lane == 0) st_relaxed_u64(&A[g], pack_state(b.epoch, kFlagAggregate, words));
+    if (lane == 0) st_relaxed_u64(&sw.A[g], pack_state(b.epoch, kFlagAggregate, words));
     if (R_l != 0u) {
       uint32_t rank = (uint32_t)__popc(bitmap & ((1u << lane) - 1u));
       atomicOr(&sm.img[rank >> 1], sz_l << (16u * (rank & 1u)));
     }
   }
+  const bool closes = (g & 31u) == 31u || g == jg.G - 1u;  // this tile completes its super-tile
+  if (closes) prefix_own_super_tile(sm, sw, g, jg.G, words, b.epoch, b.status);
   if (lg.m_blk != 0u) {
     if (lg.t == 0u) {
       or_u32(sm.img, boff, p.mu_bits);
@@ -578,7 +641,8 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const Lane
 
   // place of the group in the stream
   TL(5);
-  find_prefix(sm, A, SA, g, jg.G, words, b.epoch, b.status);
+  if (!closes) prefix_own_super_tile(sm, sw, g, jg.G, words, b.epoch, b.status);
+  prefix_earlier_super_tiles(sm, sw, g, b.epoch, b.status);
   TL(11);
   __syncthreads();
   TL(6);
@@ -610,8 +674,8 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const Lane
     if (t == 0) {
       out32[0] = kMagic;
       out32[1] = 0u;
-      out32[2] = (uint32_t)jg.len;
-      out32[3] = (uint32_t)(jg.len >> 32);
+      out32[2] = jg.len;
+      out32[3] = 0u;
       out32[4] = (uint32_t)kL;
       out32[5] = __float_as_uint(b.eb);
     }
@@ -684,10 +748,49 @@ __device__ __forceinline__ bool open_group(const uint8_t* sin, uint64_t in_bytes
   return true;
 }
 
-// sum of the 2-bit fields of a 64-bit word
-__device__ __forceinline__ uint32_t sum_fields2(uint32_t lo, uint32_t hi) {
-  return (uint32_t)(__popc(lo & 0x55555555u) + __popc(hi & 0x55555555u)) +
-         2u * (uint32_t)(__popc(lo & 0xaaaaaaaau) + __popc(hi & 0xaaaaaaaau));
+// sum of the sixteen 2-bit fields of a word
+__device__ __forceinline__ uint32_t sum_fields(uint32_t w) {
+  return (uint32_t)__popc(w & 0x55555555u) + 2u * (uint32_t)__popc(w & 0xaaaaaaaau);
+}
+
+// One byte position of a lane's summary.  The lane's 32 lead codes sit in two words (values 0-15 in lo,
+// 16-31 in hi).  Values with lead <= KB store byte KB of the field (counted from its most significant
+// byte); the last such value is found with one leading-zero count, the stored bytes before it with two
+// population counts, and its byte is fetched from the image.
+struct SummaryIn {
+  uint32_t lo, hi, lo1, hi1;  // the codes, and the codes shifted right by one
+  uint32_t vlo, vhi;          // marker bit (even positions) of every valid value
+  uint32_t lead_lo;           // sum of the leads of values 0-15
+  uint32_t B, pos0;
+};
+template <int KB>
+__device__ __forceinline__ void summary_byte(const uint32_t* img, const SummaryIn& si, uint32_t& sval, uint32_t& smask) {
+  uint32_t ph, pl;  // markers of the values that store byte KB
+  if (KB == 0) {
+    ph = ~(si.hi | si.hi1) & si.vhi;
+    pl = ~(si.lo | si.lo1) & si.vlo;
+  } else if (KB == 1) {
+    ph = ~si.hi1 & si.vhi;
+    pl = ~si.lo1 & si.vlo;
+  } else if (KB == 2) {
+    ph = ~(si.hi & si.hi1) & si.vhi;
+    pl = ~(si.lo & si.lo1) & si.vlo;
+  } else {
+    ph = si.vhi;
+    pl = si.vlo;
+  }
+  if ((ph | pl) == 0u) return;
+  const bool up = ph != 0u;
+  const uint32_t pm = up ? ph : pl, w = up ? si.hi : si.lo;
+  const uint32_t i2 = 31u - (uint32_t)__clz((int)pm);  // bit position of the value's code = 2 * (its index in the half)
+  const uint32_t below = w & ((1u << i2) - 1u);        // codes of the values before it in this half
+  const uint32_t lead_sum = (up ? si.lead_lo : 0u) + sum_fields(below);
+  const uint32_t lead_i = (w >> i2) & 3u;
+  const uint32_t i = (i2 >> 1) + (up ? 16u : 0u);
+  const uint32_t byte = img_u8(img, si.pos0 + (si.B * i - lead_sum) + ((uint32_t)KB - lead_i));
+  const uint32_t shift = 8u * (si.B - 1u - (uint32_t)KB);
+  sval |= byte << shift;
+  smask |= 0xffu << shift;
 }
 
 // One quad of the general decode path: any field width, lossless blocks, ragged slices (nvq = valid values
@@ -774,7 +877,7 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   const bool nonconst = lg.m_blk != 0u && ((map >> lg.blk) & 1u);
 
   // header, lead codes and stored-byte count of the lane
-  uint32_t R = 0u, B = 0u, code_lo = 0u, code_hi = 0u, T = 0u;
+  uint32_t R = 0u, B = 0u, code_lo = 0u, code_hi = 0u, T = 0u, lead_lo = 0u;
   const uint32_t cbytes = (lg.m_blk + 3u) >> 2;
   if (!bad && nonconst) {
     R = img_u8(img, boff + 4u);
@@ -805,39 +908,40 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
     }
     if (B == 2u && ((code_lo & (code_lo >> 1) & 0x55555555u) | (code_hi & (code_hi >> 1) & 0x55555555u)))
       bad = true;  // lead 3 cannot occur in a 2-byte field
-    T = B * lg.nv - sum_fields2(code_lo, code_hi);
+    lead_lo = sum_fields(code_lo);
+    T = B * lg.nv - lead_lo - sum_fields(code_hi);
     if (bad) T = 0u;
   }
   uint32_t total;
   const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
   if (nonconst && !bad && size_blk != 5u + cbytes + total) bad = true;
+  TL(12);
   if (__syncthreads_or(bad ? 1 : 0)) return false;
+  TL(13);
 
   // Summary of the lane's values for the predecessor chain: for each byte of the code field, the byte the
   // LAST value of the lane that stores it holds (found from the lead codes alone, then fetched).
   const uint32_t pos0 = boff + 5u + cbytes + excl;  // image offset of the lane's first stored byte
   uint32_t sval = 0u, smask = 0u;
   if (nonconst && lg.nv != 0u) {
-    const uint64_t codes = ((uint64_t)code_hi << 32) | code_lo;
-    const uint64_t kOdd = 0x5555555555555555ull;  // one marker bit per 2-bit field
-    const uint64_t f0 = codes & kOdd, f1 = (codes >> 1) & kOdd;
-    const uint64_t valid = (lg.nv < 32u ? ((1ull << (2u * lg.nv)) - 1ull) : ~0ull) & kOdd;
-#pragma unroll 1
-    for (uint32_t kb = 0; kb < B; ++kb) {
-      // values with lead <= kb store byte kb (counted from the most significant byte of the field)
-      uint64_t pm = kb == 0u ? ~(f0 | f1) : (kb == 1u ? ~f1 : (kb == 2u ? ~(f0 & f1) : ~0ull));
-      pm &= valid;
-      if (pm) {
-        const uint32_t i = (63u - (uint32_t)__clzll((long long)pm)) >> 1;  // the last such value
-        const uint64_t below = codes & ((1ull << (2u * i)) - 1ull);        // codes of the values before it
-        const uint32_t lead_sum = (uint32_t)__popcll(below & kOdd) + 2u * (uint32_t)__popcll(below & (kOdd << 1));
-        const uint32_t lead_i = (uint32_t)(codes >> (2u * i)) & 3u;
-        const uint32_t byte = img_u8(img, pos0 + (B * i - lead_sum) + (kb - lead_i));
-        const uint32_t shift = 8u * (B - 1u - kb);
-        sval |= byte << shift;
-        smask |= 0xffu << shift;
-      }
+    SummaryIn si;
+    si.lo = code_lo;
+    si.hi = code_hi;
+    si.lo1 = code_lo >> 1;
+    si.hi1 = code_hi >> 1;
+    si.vlo = 0x55555555u;  // one marker bit per valid value
+    si.vhi = 0x55555555u;
+    if (tail) {
+      si.vlo = lg.nv < 16u ? ((1u << (2u * lg.nv)) - 1u) & 0x55555555u : 0x55555555u;
+      si.vhi = lg.nv <= 16u ? 0u : (lg.nv < 32u ? ((1u << (2u * (lg.nv - 16u))) - 1u) & 0x55555555u : 0x55555555u);
     }
+    si.lead_lo = lead_lo;
+    si.B = B;
+    si.pos0 = pos0;
+    summary_byte<0>(img, si, sval, smask);
+    if (B > 1u) summary_byte<1>(img, si, sval, smask);
+    if (B > 2u) summary_byte<2>(img, si, sval, smask);
+    if (B > 3u) summary_byte<3>(img, si, sval, smask);
   }
   // carry the summaries across the quad: what a lane does not store itself comes from its left
   {
@@ -855,6 +959,7 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   }
   uint32_t prev = __shfl_up_sync(kFull, sval, 1);
   if (lg.t == 0u) prev = 0u;
+  TL(14);
 
   // the lane's 32 values
   const float mu = (lg.m_blk != 0u) ? __uint_as_float(img_u32(img, boff)) : 0.0f;
@@ -932,30 +1037,35 @@ __device__ __forceinline__ void prefetch_payload(const StreamView& sv, uint32_t 
 // bits wide: the copy starts at the 16-byte boundary at or below word a, so payload word j lands at
 // sm.img[(a & 3) + j] — decode_group reads the image through that shifted origin.
 constexpr int kStageRounds = (kMaxGroupBytes / 4 + 3 + 4 * kThreads - 1) / (4 * kThreads);  // 9
+template <int kRounds>
+__device__ __forceinline__ void stage_rounds(uint4* img4, const uint4* src4, uint32_t n4) {
+  uint4 t[kRounds];
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r)
+    if ((uint32_t)r * kThreads + threadIdx.x < n4) t[r] = __ldcs(src4 + r * kThreads + threadIdx.x);
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r)
+    if ((uint32_t)r * kThreads + threadIdx.x < n4) img4[r * kThreads + threadIdx.x] = t[r];
+}
 __device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
   const uint32_t shift = sv.a & 3u;
+  const uint32_t start = sv.a - shift;                // aligned first word
   const uint32_t n_words = sv.gw + shift;             // words to bring in, from the aligned start
-  const uint32_t* src = sv.words + (sv.base >> 2) + (sv.a - shift);
-  const uint32_t avail = sv.pw - (sv.a - shift);      // payload words from the aligned start to the stream's end
-  uint4 t[kStageRounds];
-#pragma unroll
-  for (int r = 0; r < kStageRounds; ++r) {
-    const uint32_t w = 4u * ((uint32_t)r * kThreads + threadIdx.x);
-    t[r] = make_uint4(0u, 0u, 0u, 0u);
-    if (w < n_words) {
-      if (w + 4u <= avail) {
-        t[r] = __ldcs(reinterpret_cast<const uint4*>(src + w));
-      } else {  // the very end of the stream: never read past it
-        if (w + 0u < avail) t[r].x = __ldcs(src + w + 0u);
-        if (w + 1u < avail) t[r].y = __ldcs(src + w + 1u);
-        if (w + 2u < avail) t[r].z = __ldcs(src + w + 2u);
-      }
-    }
-  }
-#pragma unroll
-  for (int r = 0; r < kStageRounds; ++r) {
-    const uint32_t w = 4u * ((uint32_t)r * kThreads + threadIdx.x);
-    if (w < n_words) *reinterpret_cast<uint4*>(&sm.img[w]) = t[r];
+  const uint32_t n4 = (n_words + 3u) >> 2;            // 16-byte pieces
+  const uint32_t* src = sv.words + (sv.base >> 2) + start;
+  if (start + 4u * n4 <= sv.pw) {                     // every piece lies inside the stream (uniform)
+    const uint4* src4 = reinterpret_cast<const uint4*>(src);
+    uint4* img4 = reinterpret_cast<uint4*>(sm.img);
+    if (n4 <= 3u * kThreads)
+      stage_rounds<3>(img4, src4, n4);
+    else if (n4 <= 5u * kThreads)
+      stage_rounds<5>(img4, src4, n4);
+    else
+      stage_rounds<kStageRounds>(img4, src4, n4);
+  } else {
+    // the last piece would reach past the end of the stream (its last group only): word by word
+#pragma unroll 4
+    for (uint32_t w = threadIdx.x; w < n_words; w += kThreads) sm.img[w] = __ldcs(src + w);
   }
 }
 
@@ -979,12 +1089,16 @@ __global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kerne
   const uint32_t rank = (uint32_t)((y + (uint32_t)b.rot) % (uint32_t)b.P);
   const float* x = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
+  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
   load_rows(rows, x, jg, g);
   prefetch_group(x, jg, g + b.prefetch_distance);
   zero_image(sm.img);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
   __syncthreads();
-  encode_group(sm, rows, lg, b, jg, g, y, sout);
+  if (tail) pad_ragged(rows, lg);
+  float mx, mn;
+  lane_minmax(reinterpret_cast<const float4*>(rows + threadIdx.x * kSliceBytes), mx, mn);
+  encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
 }
 
 __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
@@ -1002,6 +1116,8 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const float* local = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
   TL(0);
+  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
+  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
   load_rows(rows, local, jg, g);
   prefetch_group(local, jg, g + b.prefetch_distance);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
@@ -1010,7 +1126,6 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   StreamView sv;
   float4 unused[8];
-  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
   bool ok = open_group(sin, in_bytes, jg, g, sv);
   uint32_t nxt_a = 0u, nxt_e = 0u;  // directory entries of the group that will take over this SM slot
   if (ok && g + b.prefetch_distance < jg.G) {
@@ -1030,10 +1145,9 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     // a corrupt input: report it, and keep the look-back chain alive with a poisoned entry
     if (threadIdx.x == 0) {
       raise(b.status, kErrCorrupt);
-      uint64_t* A = b.tile_state + (uint64_t)y * b.state_stride;
-      st_relaxed_u64(&A[g], pack_state(b.epoch, kFlagPoison, 0));
-      if ((g & 31u) == 31u || g == jg.G - 1u)
-        st_relaxed_u64(&A[b.tiles_per_job + (g >> 5)], pack_state(b.epoch, kFlagPoison, 0));
+      const SizeWords sw = size_words(b, y);
+      st_relaxed_u64(&sw.A[g], pack_state(b.epoch, kFlagPoison, 0));
+      if ((g & 31u) == 31u || g == jg.G - 1u) st_relaxed_u64(&sw.SA[g >> 5], pack_state(b.epoch, kFlagPoison, 0));
     }
     return;
   }
@@ -1044,7 +1158,10 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     __syncthreads();  // the slices are about to be reused for staging
   }
   TL(3);
-  encode_group(sm, rows, lg, b, jg, g, y, sout);
+  if (tail) pad_ragged(rows, lg);
+  float mx, mn;
+  lane_minmax(slice, mx, mn);
+  encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
   TL(7);
 }
 

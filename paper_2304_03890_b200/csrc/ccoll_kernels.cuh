@@ -58,7 +58,7 @@ struct EncodeBatch {
   uint64_t sum_rank_stride;
   uint64_t* moved;          // nullable: += moved_mult * stream bytes of every job
   uint32_t moved_mult;
-  uint64_t* tile_state;     // size words: job y has A[tiles_per_job] then SA[ceil(tiles_per_job/32)] at y*state_stride
+  uint64_t* tile_state;     // size words of job y at y*state_stride: A[tiles], then SA[ceil(tiles/32)]
   uint32_t tiles_per_job;
   uint32_t state_stride;
   uint32_t epoch;
@@ -84,6 +84,9 @@ struct DecodeBatch {
   uint32_t prefetch_distance;  // groups ahead whose payload a CTA asks L2 for (set by the launcher)
   uint32_t* status;
 };
+
+// Size words a job of `tiles` groups needs (see tile_state).
+constexpr uint32_t state_words(uint32_t tiles) { return tiles + (tiles + 31u) / 32u; }
 
 // Each returns false if the device could not be set up (the launch was not attempted).
 bool launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);

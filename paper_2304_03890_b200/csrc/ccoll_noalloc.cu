@@ -16,7 +16,7 @@ namespace {
 using namespace ccoll;
 
 constexpr size_t kMaxGroups = CCOLL_NOALLOC_MAX_VALUES / kGroupValues;  // 16384
-constexpr size_t kSizeWords = kMaxGroups + (kMaxGroups + 31) / 32;      // A[groups] + SA[groups / 32]
+constexpr size_t kSizeWords = state_words((uint32_t)kMaxGroups);  // A[groups] + SA[groups / 32]
 
 // The scratch itself.  Every GPU that loads the library holds these ~136 KB until the process exits.
 // Zero at load time; later calls find the previous call's words in it (see the epoch below).
@@ -75,7 +75,7 @@ extern "C" int ccoll_compress_noalloc(const float* in, size_t n, float abs_err_b
   const size_t G = (((n + kL - 1) / kL) + kGroupBlocks - 1) / kGroupBlocks;
   b.tile_state = d.words;
   b.tiles_per_job = (uint32_t)G;
-  b.state_stride = (uint32_t)(G + (G + 31) / 32);
+  b.state_stride = state_words((uint32_t)G);
   b.epoch = d.epoch;
   b.status = status;
   b.eb = abs_err_bound;
