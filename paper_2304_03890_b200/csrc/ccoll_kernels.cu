@@ -160,12 +160,20 @@ struct Smem {
 constexpr int kCtlBytes = (sizeof(Smem) + 127) / 128 * 128;
 extern __shared__ __align__(128) uint8_t dyn_smem[];
 
+// The image is built with atomic ORs, so it must start as zeros.  Only its front (10 KB, more than most
+// groups need) is cleared up front; a group whose payload turns out longer clears the rest once its size is
+// known (zero_image_rest), at the price of one more barrier.
+constexpr int kZeroFrontWords = 5 * 4 * kThreads;  // five 128-bit stores per thread
+constexpr int kZeroSlackWords = 8;                 // words past the payload that placement may touch
 __device__ __forceinline__ void zero_image(uint32_t* img) {  // a barrier must follow
   uint4* p = reinterpret_cast<uint4*>(img) + threadIdx.x;
-  constexpr int kVecs = kImgWords / 4, kFullRounds = kVecs / kThreads;
 #pragma unroll
-  for (int r = 0; r < kFullRounds; ++r) p[r * kThreads] = make_uint4(0u, 0u, 0u, 0u);
-  if (kFullRounds * kThreads + (int)threadIdx.x < kVecs) p[kFullRounds * kThreads] = make_uint4(0u, 0u, 0u, 0u);
+  for (int r = 0; r < kZeroFrontWords / (4 * kThreads); ++r) p[r * kThreads] = make_uint4(0u, 0u, 0u, 0u);
+}
+__device__ __forceinline__ void zero_image_rest(uint32_t* img) {  // whole CTA; ends with a barrier
+  for (int v = kZeroFrontWords / 4 + (int)threadIdx.x; v < kImgWords / 4; v += kThreads)
+    reinterpret_cast<uint4*>(img)[v] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
 }
 
 // Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
@@ -617,6 +625,7 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const Lane
   const uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
   const uint32_t words = (raw + 3u) >> 2;
   const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
+  if (words + (uint32_t)kZeroSlackWords > (uint32_t)kZeroFrontWords) zero_image_rest(sm.img);  // rare, uniform
 
   const SizeWords sw = size_words(b, y);
   if (warp == 0) {
@@ -846,11 +855,11 @@ __device__ __forceinline__ float reduce_op(float a, float b, int op) {
 // The group's payload must already be staged in sm.img (and visible).  nblk = blocks in the group.
 // kToSlice = false: the values are returned in v[] (fully unrolled loops).  kToSlice = true (fused reduce):
 // each decoded quad is REDUCED (op) with the quad of local values waiting in the lane's slice and the result is written
-// back there; the loops are then unrolled only twice, which keeps the fused kernel inside the instruction
-// cache.
+// back there, and mx / mn receive the largest / smallest result of the lane (meaningless for a ragged slice);
+// the loops are then unrolled only twice, which keeps the fused kernel inside the instruction cache.
 template <bool kToSlice>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8], float4* slice4, int op = 0) {
+                                             float4 (&v)[8], float4* slice4, int op, float& mx, float& mn) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
@@ -967,8 +976,11 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   auto put = [&](int j, const float4& r) {
     if (kToSlice) {
       const float4 a = slice4[j];
-      slice4[j] = make_float4(reduce_op(r.x, a.x, op), reduce_op(r.y, a.y, op), reduce_op(r.z, a.z, op),
-                              reduce_op(r.w, a.w, op));
+      const float4 o = make_float4(reduce_op(r.x, a.x, op), reduce_op(r.y, a.y, op), reduce_op(r.z, a.z, op),
+                                   reduce_op(r.w, a.w, op));
+      slice4[j] = o;
+      mx = max3_nan(max3_nan(mx, o.x, o.y), o.z, o.w);  // the encoder's min/max, while the values are at hand
+      mn = min3_nan(min3_nan(mn, o.x, o.y), o.z, o.w);
     } else {
       v[j] = r;
     }
@@ -982,30 +994,32 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   const uint32_t sh = 32u - R;
   uint32_t pos = pos0;
   if (!tail && R <= 24u) {
-    // Fast path: complete slice, field of at most 3 bytes.  Shifts by computed amounts are multiplications
-    // by a power of two (FMA pipe) where the power serves twice: m = 2^(8*stored bytes) extracts the stored
-    // bytes (umulhi) and -m masks the bytes that are kept from the predecessor.
+    // Fast path: complete slice, field of at most 3 bytes.  A value is assembled by ONE byte permutation of
+    // (predecessor, next four stream bytes): it takes the top `lead` bytes of the field from the predecessor
+    // and the stored bytes, most significant first, from the stream.  The permutation depends only on the
+    // number of stored bytes nb (0..3) and is itself picked, by a byte permutation, from a two-register table.
     const uint32_t c8B = 8u * B;
     const uint32_t msh = 1u << sh;  // q << sh == q * 2^sh
+    const uint32_t kSel01 = 0x32143210u, kSel23 = 0x34563245u;  // byte selectors for nb = 0, 1 | 2, 3
+    const uint32_t kPick = 0x10u + 0x22u * B;                   // picks table entry nb = B - lead
 #pragma unroll kUnroll
     for (int j = 0; j < 8; ++j) {
       const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
-      const uint32_t c0 = c8B - 8u * (cb & 3u), c1 = c8B - 8u * ((cb >> 2) & 3u), c2 = c8B - 8u * ((cb >> 4) & 3u),
-                     c3 = c8B - 8u * (cb >> 6);
+      const uint32_t l0 = cb & 3u, l1 = (cb >> 2) & 3u, l2 = (cb >> 4) & 3u, l3 = cb >> 6;
+      const uint32_t c0 = c8B - 8u * l0, c1 = c8B - 8u * l1, c2 = c8B - 8u * l2;
       const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
       const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3];
       // at most 12 bytes per quad here: three words of string are enough
       const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z);
-      pos += (c0 + c1 + c2 + c3) >> 3;
+      pos += 4u * B - (l0 + l1 + l2 + l3);
       const uint32_t U0 = __funnelshift_r(S0, S1, c0), U1 = __funnelshift_r(S1, S2, c0);
       const uint32_t X0 = __funnelshift_r(U0, U1, c1);
       const uint32_t X1 = __funnelshift_r(U1, S2 >> c0, c1);
       const uint32_t r3 = __funnelshift_r(X0, X1, c2);
-      const uint32_t m0 = 1u << c0, m1 = 1u << c1, m2 = 1u << c2, m3 = 1u << c3;
-      const uint32_t q0 = __umulhi(__byte_perm(S0, 0u, 0x0123), m0) | (prev & (0u - m0));
-      const uint32_t q1 = __umulhi(__byte_perm(U0, 0u, 0x0123), m1) | (q0 & (0u - m1));
-      const uint32_t q2 = __umulhi(__byte_perm(X0, 0u, 0x0123), m2) | (q1 & (0u - m2));
-      const uint32_t q3 = __umulhi(__byte_perm(r3, 0u, 0x0123), m3) | (q2 & (0u - m3));
+      const uint32_t q0 = __byte_perm(prev, S0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l0));
+      const uint32_t q1 = __byte_perm(q0, U0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l1));
+      const uint32_t q2 = __byte_perm(q1, X0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l2));
+      const uint32_t q3 = __byte_perm(q2, r3, __byte_perm(kSel01, kSel23, kPick - 0x22u * l3));
       prev = q3;
       put(j, make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
                          __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu)));
@@ -1126,6 +1140,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   StreamView sv;
   float4 unused[8];
+  float mx = __uint_as_float(0xff800000u), mn = __uint_as_float(0x7f800000u);  // -inf, +inf
   bool ok = open_group(sin, in_bytes, jg, g, sv);
   uint32_t nxt_a = 0u, nxt_e = 0u;  // directory entries of the group that will take over this SM slot
   if (ok && g + b.prefetch_distance < jg.G) {
@@ -1138,7 +1153,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     __syncthreads();  // the image and the local values in the rows are complete
     TL(1);
     // decoded + local, one rounded add per value, left in the lane's slice
-    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice, b.op);
+    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice, b.op, mx, mn);
   }
   TL(2);
   if (!ok) {
@@ -1158,9 +1173,10 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     __syncthreads();  // the slices are about to be reused for staging
   }
   TL(3);
-  if (tail) pad_ragged(rows, lg);
-  float mx, mn;
-  lane_minmax(slice, mx, mn);
+  if (tail) {
+    pad_ragged(rows, lg);
+    lane_minmax(slice, mx, mn);
+  }
   encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
   TL(7);
 }
@@ -1195,7 +1211,8 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
     prefetch_payload(sv, nxt_a, nxt_e);
     __syncthreads();
     TL(2);
-    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr);
+    float mx_unused, mn_unused;
+    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr, 0, mx_unused, mn_unused);
   }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
