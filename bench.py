@@ -33,13 +33,13 @@ SIGMA = 8.0
 P_SIM = 8
 METRIC = "compress / decompress / fused reduce-step GB/s (fp32 input) and % of B200 HBM peak"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of each kernel on the
-# 256x512x256 field of the same recipe (33,554,432 values; profiles/kernels_256x512x256_four_lanes_per_block.md),
+# 256x512x256 field of the same recipe (33,554,432 values; profiles/kernels_256x512x256.md),
 # expressed per value: DRAM traffic grows in proportion to the values processed, so a full-size launch is
 # this figure times its value count.  (Writes that are still in L2 when the kernel ends are not in it.)
 NCU_DRAM_BYTES_PER_VALUE = {
-    "ccoll_compress_kernel": (134.33e6 + 8.64e6) / 33554432,
-    "ccoll_decode_kernel": (58.71e6 + 76.01e6) / 33554432,
-    "ccoll_reduce_kernel": (193.06e6 + 150.80e6) / 33554432,
+    "ccoll_compress_kernel": (134.29e6 + 6.97e6) / 33554432,
+    "ccoll_decode_kernel": (58.71e6 + 76.52e6) / 33554432,
+    "ccoll_reduce_kernel": (193.10e6 + 151.46e6) / 33554432,
 }
 
 
