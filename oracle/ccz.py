@@ -9,7 +9,7 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_CORRUPT = 0, 1, 3, 4
 BLOCK_CONSTANT, BLOCK_TRUNCATED, BLOCK_LOSSLESS = 0, 1, 2
-OP_SUM, OP_MAX, OP_MIN = 0, 1, 2
+OP_SUM, OP_MAX, OP_MIN, OP_AVG = 0, 1, 2, 3
 
 _lib = None
 

@@ -449,8 +449,9 @@ int ccz_reduce_step(const uint8_t* in, size_t in_bytes, const float* local, size
  *   MAX: a (the decoded value) if a > b or b is a NaN, else b (the local value); a pure selection, so the
  *        result is one of the two bit patterns.  MIN likewise with <.  (With equal values, e.g. -0 and
  *        +0, the local value is taken.) */
-int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L, int op,
-                       uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
+/* decode, reduce with the local chunk, optionally divide by `divisor` (0 = no division), encode */
+static int reduce_round(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L, int op,
+                        float divisor, uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
   if (!local && n) return CCZ_ERR_INVALID_ARG;
   if (op != CCZ_OP_SUM && op != CCZ_OP_MAX && op != CCZ_OP_MIN) return CCZ_ERR_INVALID_ARG;
   std::vector<float> s(n);
@@ -460,6 +461,7 @@ int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, s
     float a = s[i], b = local[i], t;
     if (op == CCZ_OP_SUM) {
       t = a + b;
+      if (divisor != 0.0f) t = t / divisor; /* Average = Sum whose last round divides by the rank count */
       if (t != t) t = float_of(0x7FFFFFFFu);
     } else if (op == CCZ_OP_MAX) {
       t = (a > b || b != b) ? a : b;
@@ -475,6 +477,11 @@ int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, s
   return CCZ_OK;
 }
 
+int ccz_reduce_step_op(const uint8_t* in, size_t in_bytes, const float* local, size_t n, float eb, uint32_t L, int op,
+                       uint8_t* out, size_t cap, uint64_t* out_bytes, float* sum_out) {
+  return reduce_round(in, in_bytes, local, n, eb, L, op, 0.0f, out, cap, out_bytes, sum_out);
+}
+
 int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, uint32_t L, uint64_t* bytes_moved) {
   return ccz_allreduce_sim_op(in, out, P, n, eb, L, CCZ_OP_SUM, bytes_moved);
 }
@@ -482,8 +489,12 @@ int ccz_allreduce_sim(const float* in, float* out, int P, size_t n, float eb, ui
 int ccz_allreduce_sim_op(const float* in, float* out, int P, size_t n, float eb, uint32_t L, int op,
                          uint64_t* bytes_moved) {
   if (P < 1 || ((!in || !out) && n)) return CCZ_ERR_INVALID_ARG;
-  if (op != CCZ_OP_SUM && op != CCZ_OP_MAX && op != CCZ_OP_MIN) return CCZ_ERR_INVALID_ARG;
+  if (op != CCZ_OP_SUM && op != CCZ_OP_MAX && op != CCZ_OP_MIN && op != CCZ_OP_AVG) return CCZ_ERR_INVALID_ARG;
   if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  /* Average (Sec. III-B, the corollary after Theorem 1): the ring adds as for Sum; the chunk's owner, who
+   * forms the complete sum in the last round, divides it by the number of ranks before it is compressed
+   * for the allgather. */
+  const int step_op = op == CCZ_OP_AVG ? CCZ_OP_SUM : op;
   size_t C = ccz_chunk_len(n, P, L);
   uint64_t moved = 0;
   std::vector<uint8_t> sa, sb;
@@ -511,8 +522,9 @@ int ccz_allreduce_sim_op(const float* in, float* out, int P, size_t n, float eb,
       int r = (c + k) % P;
       uint64_t nbytes = 0;
       float* sum_out = (k == P - 1) ? out + (size_t)owner * n + lo : nullptr;
-      rc = ccz_reduce_step_op(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, op, sb.data(), cap,
-                              &nbytes, sum_out);
+      const float divisor = (op == CCZ_OP_AVG && k == P - 1) ? (float)P : 0.0f;
+      rc = reduce_round(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, step_op, divisor, sb.data(), cap,
+                        &nbytes, sum_out);
       if (rc != CCZ_OK) return rc;
       sa.swap(sb);
       bytes = nbytes;

@@ -47,7 +47,8 @@ enum {
 };
 
 enum { CCZ_BLOCK_CONSTANT = 0, CCZ_BLOCK_TRUNCATED = 1, CCZ_BLOCK_LOSSLESS = 2 };
-enum { CCZ_OP_SUM = 0, CCZ_OP_MAX = 1, CCZ_OP_MIN = 2 }; /* reductions analysed in Sec. III-B */
+enum { CCZ_OP_SUM = 0, CCZ_OP_MAX = 1, CCZ_OP_MIN = 2, CCZ_OP_AVG = 3 }; /* reductions analysed in Sec. III-B;
+                                                                          AVG only in the all-reduce replay */
 
 /* Worst-case stream size for n values in blocks of block_len. */
 size_t ccz_compress_bound(size_t n, uint32_t block_len);

@@ -178,3 +178,52 @@ def test_max_min_equal_values_take_the_local_one():
         assert total.tobytes() == b.tobytes()
     with pytest.raises(ccz.OracleError):
         ccz.reduce_step(s0, b, np.float32(1e-3), op=7)
+
+
+# ---- Average (Sec. III-B, the corollary after Theorem 1): Sum whose owner divides by the rank count ----
+def chunk_bounds(n, P, c):
+    C = -(-(-(-n // P)) // 128) * 128      # ceil(ceil(n / P) / 128) * 128
+    return min(c * C, n), min((c + 1) * C, n)
+
+
+@pytest.mark.parametrize("P,n", [(2, 5000), (3, 4096 * 3), (4, 128 * 37 + 5), (8, 24 * 24 * 32)])
+def test_average_is_the_owners_sum_divided_once(P, n):
+    rng = np.random.default_rng(100 + P)
+    x = (rng.standard_normal((P, n)) * 3).astype(np.float32)
+    eb = np.float32(1e-2)
+    s, moved_sum = ccz.allreduce_sim(x, eb, op=ccz.OP_SUM)
+    a, moved_avg = ccz.allreduce_sim(x, eb, op=ccz.OP_AVG)
+    for c in range(P):
+        lo, hi = chunk_bounds(n, P, c)
+        if hi == lo:
+            continue
+        owner = (c - 1) % P
+        # the owner holds the complete, uncompressed sum: its average is that sum divided once, in fp32
+        want = (s[owner, lo:hi] / np.float32(P)).astype(np.float32)
+        assert a[owner, lo:hi].tobytes() == want.tobytes()
+        # every other rank holds that average after one compression
+        dec = ccz.decompress(ccz.compress(want, eb), hi - lo)
+        for r in range(P):
+            if r != owner:
+                assert a[r, lo:hi].tobytes() == dec.tobytes()
+    # error law: (P-1) lossy rounds before the division, one after it
+    mean = x.astype(np.float64).mean(axis=0)
+    bound = ((P - 1) / P + 1) * float(eb) + 2.0 ** -22 * np.abs(x).sum(axis=0).max()
+    assert np.abs(a - mean).max() <= bound
+
+
+def test_average_special_cases():
+    eb = np.float32(1e-3)
+    x = np.linspace(-1, 1, 700, dtype=np.float32)[None, :]
+    a, moved = ccz.allreduce_sim(x, eb, op=ccz.OP_AVG)          # one rank: nothing moves, x / 1 == x
+    assert a.tobytes() == x.tobytes() and moved == 0
+    # constant blocks of small integers: every sum and the division are exact
+    P, n = 4, 128 * 6
+    base = np.repeat(np.arange(6, dtype=np.float32) * 4, 128)
+    ranks = np.stack([base + 4 * r for r in range(P)]).astype(np.float32)
+    a, _ = ccz.allreduce_sim(ranks, eb, op=ccz.OP_AVG)
+    assert np.array_equal(a, np.broadcast_to(base + 6, (P, n)))
+    # a NaN average is the canonical quiet NaN
+    ranks[1, 5] = np.nan
+    a, _ = ccz.allreduce_sim(ranks, eb, op=ccz.OP_AVG)
+    assert (a.view(np.uint32)[:, 5] == 0x7FFFFFFF).all()
