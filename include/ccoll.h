@@ -62,7 +62,8 @@ typedef enum {
 #define CCOLL_MAX_VALUES ((size_t)1 << 29) /* values per stream (2 GiB of fp32) */
 
 enum { CCOLL_BCAST = 0, CCOLL_SCATTER = 1 };
-enum { CCOLL_SUM = 0, CCOLL_MAX = 1, CCOLL_MIN = 2 }; /* reductions of the computation framework, Sec. III-B */
+enum { CCOLL_SUM = 0, CCOLL_MAX = 1, CCOLL_MIN = 2, CCOLL_AVG = 3 }; /* reductions of the computation framework,
+                                                                         Sec. III-B; AVG only in ccoll_allreduce_sim_op */
 
 /* Worst-case stream size in bytes for n values (0 if block_len is unsupported).  Output buffers of
  * ccoll_compress / ccoll_reduce_step must hold this many bytes. */
@@ -130,7 +131,10 @@ int ccoll_reduce_step_op(const void* in, size_t in_bytes, const float* local, si
 int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
                         uint64_t* bytes_moved, void* stream);
 
-/* ccoll_allreduce_sim with the reduction chosen (CCOLL_SUM / CCOLL_MAX / CCOLL_MIN, as ccoll_reduce_step_op). */
+/* ccoll_allreduce_sim with the reduction chosen: CCOLL_SUM / CCOLL_MAX / CCOLL_MIN as in ccoll_reduce_step_op, or
+ * CCOLL_AVG (Sec. III-B, the corollary after Theorem 1): the ring adds as for Sum, and the chunk's owner, in the
+ * round that completes the sum, divides it by P (one correctly rounded fp32 division; a NaN quotient is
+ * 0x7FFFFFFF) before it is compressed for the allgather.  The owner keeps the uncompressed average. */
 int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
                            int op, uint64_t* bytes_moved, void* stream);
 

@@ -12,7 +12,7 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_CORRUPT, ERR_TIMEOUT, ERR_CUDA = range(7)
 BCAST, SCATTER = 0, 1
-SUM, MAX, MIN = 0, 1, 2
+SUM, MAX, MIN, AVG = 0, 1, 2, 3
 BLOCK_LEN = 128
 _NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CAPACITY", 4: "CORRUPT", 5: "TIMEOUT", 6: "CUDA"}
 

@@ -229,7 +229,7 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
 int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
                            int op, uint64_t* bytes_moved, void* stream) {
   if (P < 1 || (size_t)P > kMaxJobs) return CCOLL_ERR_INVALID_ARG;
-  if (op != CCOLL_SUM && op != CCOLL_MAX && op != CCOLL_MIN) return CCOLL_ERR_INVALID_ARG;
+  if (op != CCOLL_SUM && op != CCOLL_MAX && op != CCOLL_MIN && op != CCOLL_AVG) return CCOLL_ERR_INVALID_ARG;
   size_t C = ccoll_chunk_len(n, P, block_len);
   int rc = check_common(C, abs_err_bound, block_len);
   if (rc != CCOLL_OK) return rc;
@@ -262,7 +262,9 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
     b.n = n;
     b.P = P;
     b.rot = k;  // in round k, chunk c is at rank (c + k) mod P
-    b.op = op;
+    // Average: the ring adds; the owner's round (the last) also divides the complete sum by the rank count
+    b.op = op == CCOLL_AVG ? (k == P - 1 ? 3 : CCOLL_SUM) : op;
+    b.divisor = (float)P;
     b.s_stride = S;
     b.out_cap = S;
     b.moved = bytes_moved;

@@ -844,8 +844,15 @@ __device__ __noinline__ float4 decode_quad_generic(const uint32_t* img, DecodeCu
 
 // One reduction of the collective-computation framework (Sec. III-B): a = decoded value, b = local value.
 // Sum: one rounded add (a NaN result is the GPU's canonical 0x7FFFFFFF).  Max / Min: a pure selection, a if
-// it beats b or b is a NaN, else b.
-__device__ __forceinline__ float reduce_op(float a, float b, int op) {
+// it beats b or b is a NaN, else b.  kDivide (the owner's round of an Average, a kernel of its own so that the
+// division costs the other rounds nothing): the sum, then one correctly rounded division by the number of
+// ranks; a NaN quotient is made the same canonical NaN.
+template <bool kDivide>
+__device__ __forceinline__ float reduce_op(float a, float b, int op, float divisor) {
+  if (kDivide) {
+    const float q = __fdiv_rn(__fadd_rn(a, b), divisor);
+    return q != q ? __uint_as_float(0x7fffffffu) : q;
+  }
   if (op == 0) return __fadd_rn(a, b);
   if (op == 1) return (a > b || b != b) ? a : b;
   return (a < b || b != b) ? a : b;
@@ -857,9 +864,10 @@ __device__ __forceinline__ float reduce_op(float a, float b, int op) {
 // each decoded quad is REDUCED (op) with the quad of local values waiting in the lane's slice and the result is written
 // back there, and mx / mn receive the largest / smallest result of the lane (meaningless for a ragged slice);
 // the loops are then unrolled only twice, which keeps the fused kernel inside the instruction cache.
-template <bool kToSlice>
+template <bool kToSlice, bool kDivide = false>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8], float4* slice4, int op, float& mx, float& mn) {
+                                             float4 (&v)[8], float4* slice4, int op, float divisor, float& mx,
+                                             float& mn) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
@@ -976,8 +984,8 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   auto put = [&](int j, const float4& r) {
     if (kToSlice) {
       const float4 a = slice4[j];
-      const float4 o = make_float4(reduce_op(r.x, a.x, op), reduce_op(r.y, a.y, op), reduce_op(r.z, a.z, op),
-                                   reduce_op(r.w, a.w, op));
+      const float4 o = make_float4(reduce_op<kDivide>(r.x, a.x, op, divisor), reduce_op<kDivide>(r.y, a.y, op, divisor),
+                                   reduce_op<kDivide>(r.z, a.z, op, divisor), reduce_op<kDivide>(r.w, a.w, op, divisor));
       slice4[j] = o;
       mx = max3_nan(max3_nan(mx, o.x, o.y), o.z, o.w);  // the encoder's min/max, while the values are at hand
       mn = min3_nan(min3_nan(mn, o.x, o.y), o.z, o.w);
@@ -1115,6 +1123,7 @@ __global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kerne
   encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
 }
 
+template <bool kDivide>
 __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
@@ -1153,7 +1162,8 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     __syncthreads();  // the image and the local values in the rows are complete
     TL(1);
     // decoded + local, one rounded add per value, left in the lane's slice
-    ok = decode_group<true>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice, b.op, mx, mn);
+    ok = decode_group<true, kDivide>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice,
+                                     b.op, b.divisor, mx, mn);
   }
   TL(2);
   if (!ok) {
@@ -1212,7 +1222,7 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
     __syncthreads();
     TL(2);
     float mx_unused, mn_unused;
-    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr, 0, mx_unused, mn_unused);
+    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr, 0, 0.0f, mx_unused, mn_unused);
   }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
@@ -1243,7 +1253,8 @@ bool device_ready() {
   if (!g_ready[dev]) {
     int sms = 0, per_sm = 0;
     if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(ccoll_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(ccoll_reduce_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(ccoll_reduce_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDecode) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_compress_kernel, kThreads, kSmemBytes) != cudaSuccess)
@@ -1277,7 +1288,10 @@ bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cu
 bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
   const EncodeBatch b = with_prefetch(b0, jobs);
-  ccoll_reduce_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+  if (b.op == 3)
+    ccoll_reduce_kernel<true><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+  else
+    ccoll_reduce_kernel<false><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
   return true;
 }
 bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {

@@ -46,7 +46,8 @@ struct EncodeBatch {
   uint64_t chunk_len;       // C
   uint64_t n;               // values per rank buffer
   int P, rot;
-  int op;                   // reduce step only: 0 sum, 1 max, 2 min
+  int op;                   // reduce step only: 0 sum, 1 max, 2 min, 3 sum then division by `divisor`
+  float divisor;            // op 3 only (the last round of an Average: the number of ranks)
   const uint8_t* sin;       // incoming streams (reduce step only), job y at sin + y*s_stride
   const uint64_t* sin_bytes;  // device array indexed by job, or null -> sin_bytes_host
   uint64_t sin_bytes_host;

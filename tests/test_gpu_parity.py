@@ -286,3 +286,23 @@ def test_max_min_reduce_step_and_allreduce_match_oracle(op):
     with pytest.raises(B.CcollError) as e:
         B.reduce_step(dev(s0), dev(b_), eb, op=5)
     assert e.value.code == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("P,n", [(1, 700), (2, 128 * 37 + 4), (3, 4096 * 3), (8, 32 * 32 * 40)])
+def test_average_allreduce_matches_oracle(P, n):
+    rng = np.random.default_rng(300 + P)
+    xs = (rng.standard_normal((P, n)) * 5).astype(np.float32)
+    xs[0, 3] = np.float32(1e-41)            # a denormal: the division is correctly rounded there too
+    if P > 1:
+        xs[1, n // 2] = np.nan              # a NaN average is the canonical quiet NaN
+        xs[P - 1, 128:256] = 7.0            # constant blocks stay exact
+        xs[:P - 1, 128:256] = 1.0
+    eb = 2e-2
+    ref, ref_moved = ccz.allreduce_sim(xs, eb, op=ccz.OP_AVG)
+    got, moved = B.allreduce_sim(dev(xs), eb, op=B.AVG)
+    assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
+    # the step-level entry point has no rank count to divide by
+    s0 = ccz.compress(xs[0], eb)
+    with pytest.raises(B.CcollError) as e:
+        B.reduce_step(dev(s0), dev(xs[0]), eb, op=B.AVG)
+    assert e.value.code == B.ERR_INVALID_ARG
