@@ -42,6 +42,10 @@ def lib():
         L.ccz_allreduce_sim_op.argtypes = [vp, vp, i32, sz, f32, u32, i32, vp]
         L.ccz_bcast_sim.restype = i32
         L.ccz_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp]
+        L.ccz_bcast_sim_p2p.restype = i32
+        L.ccz_bcast_sim_p2p.argtypes = [vp, vp, sz, i32, sz, f32, u32, vp]
+        L.ccz_allreduce_sim_p2p.restype = i32
+        L.ccz_allreduce_sim_p2p.argtypes = [vp, vp, i32, sz, f32, u32, vp]
         _lib = L
     return _lib
 
@@ -132,3 +136,23 @@ def bcast_sim(root, P, eb, block_len=128, mode=0):
     cb = np.zeros(P, dtype=np.uint64)
     _check(lib().ccz_bcast_sim(_ptr(root), _ptr(out), stride, P, n, eb, block_len, mode, _ptr(cb)))
     return out, cb
+
+
+def bcast_sim_p2p(root, P, eb, block_len=128):
+    """CPR-P2P broadcast over the binomial tree.  Returns (out [P, n], hops [P])."""
+    root = _f32(root)
+    n = root.size
+    out = np.zeros((P, n), dtype=np.float32)
+    hops = np.zeros(P, dtype=np.uint32)
+    _check(lib().ccz_bcast_sim_p2p(_ptr(root), _ptr(out), n, P, n, eb, block_len, _ptr(hops)))
+    return out, hops
+
+
+def allreduce_sim_p2p(x, eb, block_len=128):
+    """CPR-P2P all-reduce (Sum).  x: [P, n] fp32.  Returns (out [P, n], bytes_moved)."""
+    x = _f32(x)
+    P, n = x.shape
+    out = np.zeros((P, n), dtype=np.float32)
+    moved = ctypes.c_uint64(0)
+    _check(lib().ccz_allreduce_sim_p2p(_ptr(x), _ptr(out), P, n, eb, block_len, ctypes.byref(moved)))
+    return out, int(moved.value)

@@ -579,4 +579,83 @@ int ccz_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int 
   return CCZ_OK;
 }
 
+/* ---- CPR-P2P replays: what the frameworks are compared with (Sec. III-A-1, III-A-2) ---- */
+
+/* one hop of a compression-enabled point-to-point transfer: the sender compresses, the receiver decompresses */
+static int p2p_hop(const float* src, size_t len, float eb, uint32_t L, float* dst, uint64_t* bytes) {
+  size_t cap = ccz_compress_bound(len, L);
+  std::vector<uint8_t> stream(cap, 0);
+  uint64_t nb = 0;
+  int rc = ccz_compress(src, len, eb, L, stream.data(), cap, &nb);
+  if (rc != CCZ_OK) return rc;
+  if (bytes) *bytes += nb;
+  return ccz_decompress(stream.data(), (size_t)nb, len, L, dst);
+}
+
+int ccz_bcast_sim_p2p(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float eb, uint32_t L,
+                      uint32_t* hops) {
+  if (P < 1 || ((!root_in || !out) && n) || (P > 1 && out_rank_stride < n)) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  /* binomial tree rooted at rank 0: in round k every rank r < 2^k sends to rank r + 2^k, so rank r > 0
+   * receives from r with its highest set bit cleared, and what it receives has been compressed and
+   * decompressed once more than its parent's copy */
+  for (size_t i = 0; i < n; ++i) out[i] = root_in[i];
+  if (hops) hops[0] = 0;
+  for (int r = 1; r < P; ++r) {
+    int top = 1;
+    while (top * 2 <= r) top *= 2;
+    int parent = r - top;
+    int rc = p2p_hop(out + (size_t)parent * out_rank_stride, n, eb, L, out + (size_t)r * out_rank_stride, nullptr);
+    if (rc != CCZ_OK) return rc;
+    if (hops) hops[r] = hops[parent] + 1;
+  }
+  return CCZ_OK;
+}
+
+int ccz_allreduce_sim_p2p(const float* in, float* out, int P, size_t n, float eb, uint32_t L, uint64_t* bytes_moved) {
+  if (P < 1 || ((!in || !out) && n)) return CCZ_ERR_INVALID_ARG;
+  if (!valid_block_len(L) || !valid_eb(eb)) return CCZ_ERR_INVALID_ARG;
+  size_t C = ccz_chunk_len(n, P, L);
+  uint64_t moved = 0;
+  std::vector<uint8_t> sa, sb;
+  for (int c = 0; c < P; ++c) {
+    size_t lo = (size_t)c * C < n ? (size_t)c * C : n;
+    size_t hi = (size_t)(c + 1) * C < n ? (size_t)(c + 1) * C : n;
+    size_t len = hi - lo;
+    if (P == 1) {
+      for (size_t i = 0; i < len; ++i) out[lo + i] = in[lo + i];
+      continue;
+    }
+    /* reduce-scatter: every hop compresses anyway, so it is the ring of Fig. 4 */
+    size_t cap = ccz_compress_bound(len, L);
+    sa.assign(cap, 0);
+    sb.assign(cap, 0);
+    uint64_t bytes = 0;
+    int rc = ccz_compress(in + (size_t)c * n + lo, len, eb, L, sa.data(), cap, &bytes);
+    if (rc != CCZ_OK) return rc;
+    moved += bytes;
+    int owner = (c + P - 1) % P;
+    for (int k = 1; k <= P - 1; ++k) {
+      int r = (c + k) % P;
+      uint64_t nbytes = 0;
+      float* sum_out = (k == P - 1) ? out + (size_t)owner * n + lo : nullptr;
+      rc = reduce_round(sa.data(), (size_t)bytes, in + (size_t)r * n + lo, len, eb, L, CCZ_OP_SUM, 0.0f, sb.data(), cap,
+                        &nbytes, sum_out);
+      if (rc != CCZ_OK) return rc;
+      sa.swap(sb);
+      bytes = nbytes;
+      if (k < P - 1) moved += bytes;
+    }
+    /* ring allgather with a compression at every hop: the rank h hops behind the owner receives what its
+     * predecessor holds, compressed and decompressed once more */
+    for (int h = 1; h <= P - 1; ++h) {
+      int src = (owner + h - 1) % P, dst = (owner + h) % P;
+      rc = p2p_hop(out + (size_t)src * n + lo, len, eb, L, out + (size_t)dst * n + lo, &moved);
+      if (rc != CCZ_OK) return rc;
+    }
+  }
+  if (bytes_moved) *bytes_moved = moved;
+  return CCZ_OK;
+}
+
 } /* extern "C" */

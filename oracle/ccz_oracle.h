@@ -98,6 +98,19 @@ int ccz_allreduce_sim_op(const float* in, float* out, int P, size_t n, float eb,
 int ccz_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float eb,
                   uint32_t block_len, int mode, uint64_t* chunk_bytes);
 
+/* What the frameworks are compared with: CPR-P2P, compression-enabled point-to-point transfers, where every
+ * hop compresses before sending and decompresses on arrival (Sec. III-A-1).
+ * Broadcast over the binomial tree rooted at rank 0 (Fig. 3): rank r receives from r with its highest set bit
+ * cleared; out as in ccz_bcast_sim (BCAST), out_rank_stride >= n; hops (nullable, [P]) = tree depth of a rank. */
+int ccz_bcast_sim_p2p(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float eb,
+                      uint32_t block_len, uint32_t* hops);
+
+/* All-reduce (Sum) whose allgather stage recompresses at every hop of the ring (Fig. 2, upper half): the rank h
+ * hops behind a chunk's owner holds the owner's sum after h compress/decompress pairs.  The reduce-scatter is
+ * the ring of ccz_allreduce_sim.  bytes_moved counts every hop's stream once. */
+int ccz_allreduce_sim_p2p(const float* in, float* out, int P, size_t n, float eb, uint32_t block_len,
+                          uint64_t* bytes_moved);
+
 #ifdef __cplusplus
 }
 #endif

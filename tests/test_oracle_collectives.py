@@ -227,3 +227,68 @@ def test_average_special_cases():
     ranks[1, 5] = np.nan
     a, _ = ccz.allreduce_sim(ranks, eb, op=ccz.OP_AVG)
     assert (a.view(np.uint32)[:, 5] == 0x7FFFFFFF).all()
+
+
+# ---- CPR-P2P replays (Sec. III-A-1): a compression at every hop, the behaviour the frameworks remove ----
+def dc(x, eb):
+    return ccz.decompress(ccz.compress(x, eb), x.size)
+
+
+@pytest.mark.parametrize("P", [1, 2, 5, 8, 13])
+def test_p2p_bcast_recompresses_along_the_binomial_tree(P):
+    x = fields.config1(n=128 * 41 + 7)["x"].numpy()
+    eb = np.float32(fields.config1(n=128 * 41 + 7)["eb"])
+    out, hops = ccz.bcast_sim_p2p(x, P, eb)
+    assert [int(h) for h in hops] == [bin(r).count("1") for r in range(P)]   # depth in a binomial tree
+    assert out[0].tobytes() == x.tobytes()
+    # independent restatement: depth d holds (decompress o compress)^d (x); depth 1 is the framework's result
+    level = [x]
+    for d in range(1, int(hops.max()) + 1):
+        level.append(dc(level[-1], eb))
+    for r in range(P):
+        assert out[r].tobytes() == level[hops[r]].tobytes()
+        assert np.abs(out[r].astype(np.float64) - x).max() <= int(hops[r]) * float(eb) * (1 + 1e-6)
+    if P > 1:
+        frame, _ = ccz.bcast_sim(x, P, eb, mode=0)
+        assert out[1].tobytes() == frame[1].tobytes()
+        # the error does grow with depth on this input: what compress-once avoids
+        errs = [np.sqrt(((level[d].astype(np.float64) - x) ** 2).mean()) for d in range(len(level))]
+        assert all(errs[d + 1] >= errs[d] for d in range(len(errs) - 1))
+        if len(errs) > 2:
+            assert errs[2] > 1.1 * errs[1]                                   # RMS error, second hop
+
+
+def test_p2p_bcast_constant_blocks_survive_any_depth():
+    x = np.repeat(np.arange(9, dtype=np.float32) * 0.5, 128)
+    out, hops = ccz.bcast_sim_p2p(x, 16, np.float32(1e-3))
+    assert np.array_equal(out, np.broadcast_to(x, (16, x.size)))
+
+
+@pytest.mark.parametrize("P,n", [(1, 900), (2, 5000), (4, 128 * 37 + 5), (8, 24 * 24 * 32)])
+def test_p2p_allreduce_recompresses_along_the_allgather_ring(P, n):
+    x, eb = ranks_c3(max(P, 2))
+    x = np.ascontiguousarray(x[:P, :n])
+    got, moved = ccz.allreduce_sim_p2p(x, eb)
+    ref, ref_moved = ccz.allreduce_sim(x, eb)
+    if P == 1:
+        assert got.tobytes() == x.tobytes() and moved == 0
+        return
+    exact = x.astype(np.float64).sum(axis=0)
+    total_moved = 0
+    for c in range(P):
+        lo, hi = chunk_bounds(n, P, c)
+        if hi == lo:
+            continue
+        owner = (c - 1) % P
+        # the reduce-scatter is the same ring: owner and its first successor agree with the framework's replay
+        assert got[owner, lo:hi].tobytes() == ref[owner, lo:hi].tobytes()
+        assert got[(owner + 1) % P, lo:hi].tobytes() == ref[(owner + 1) % P, lo:hi].tobytes()
+        held = got[owner, lo:hi]
+        for h in range(1, P):
+            held = dc(held, eb)                                     # one more compression per hop
+            r = (owner + h) % P
+            assert got[r, lo:hi].tobytes() == held.tobytes()
+            bound = (P - 1 + h) * float(eb) + 2.0 ** -22 * np.abs(x[:, lo:hi]).sum(axis=0).max()
+            assert np.abs(held - exact[lo:hi]).max() <= bound
+    # same number of transfers as the framework's replay, every one carrying a freshly compressed stream
+    assert moved > 0 and abs(moved - ref_moved) <= 0.05 * ref_moved
