@@ -149,6 +149,27 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
 int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n,
                     float abs_err_bound, uint32_t block_len, int mode, uint64_t* chunk_bytes, void* stream);
 
+/* What the frameworks are compared with (Sec. III-A-1): CPR-P2P, compression-enabled point-to-point
+ * transfers, where every hop compresses before sending and decompresses on arrival.  The two replays below
+ * exist to measure what compress-once removes: the repeated compression work and the growth of the error
+ * with the number of hops.
+ *
+ * Broadcast over the binomial tree rooted at rank 0 (Fig. 3): rank r receives from r with its highest set bit
+ * cleared, so its copy has gone through popcount(r) compress/decompress pairs (rank 0: exact copy).
+ *   root_in [n] fp32;  out: rank r's n values start at out + r*out_rank_stride (floats, >= n, multiple of 4);
+ *   must not alias root_in.  Workspace as for ccoll_bcast_sim.  Ranks of equal depth hold equal data, so the
+ *   replay runs one batched compress + decode per depth (ceil(log2 P) of them) and copies. */
+int ccoll_bcast_sim_p2p(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n,
+                        float abs_err_bound, uint32_t block_len, void* stream);
+
+/* All-reduce (Sum) whose allgather recompresses at every hop of the ring (Fig. 2, upper half).  The
+ * reduce-scatter is that of ccoll_allreduce_sim (every round compresses in either scheme).  Then the rank h
+ * hops behind a chunk's owner (h = 1 .. P-1) receives what its predecessor holds, compressed and decompressed
+ * once more; the owner keeps the uncompressed sum.  Arguments as ccoll_allreduce_sim; bytes_moved counts
+ * every hop's stream once.  Launches: 1 compress, P-1 fused rounds, then P-1 decodes and P-2 compresses. */
+int ccoll_allreduce_sim_p2p(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                            uint64_t* bytes_moved, void* stream);
+
 /* ccoll_compress for callers that cannot give the library scratch memory.  (No counterpart in the paper: it
  * is a packaging of ccoll_compress, not a step of the method.)
  *

@@ -18,7 +18,8 @@ _NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CAPACITY", 4: "CORRUP
 
 EXPORTS = ("ccoll_compress_bound", "ccoll_chunk_len", "ccoll_workspace_bytes", "ccoll_set_workspace",
            "ccoll_get_status", "ccoll_compress", "ccoll_decompress", "ccoll_reduce_step", "ccoll_allreduce_sim",
-           "ccoll_bcast_sim", "ccoll_compress_noalloc", "ccoll_reduce_step_op", "ccoll_allreduce_sim_op")
+           "ccoll_bcast_sim", "ccoll_compress_noalloc", "ccoll_reduce_step_op", "ccoll_allreduce_sim_op",
+           "ccoll_bcast_sim_p2p", "ccoll_allreduce_sim_p2p")
 
 _lib = None
 
@@ -56,6 +57,10 @@ def lib():
     L.ccoll_allreduce_sim.argtypes = [vp, vp, i32, sz, f32, u32, vp, vp]
     L.ccoll_bcast_sim.restype = i32
     L.ccoll_bcast_sim.argtypes = [vp, vp, sz, i32, sz, f32, u32, i32, vp, vp]
+    L.ccoll_bcast_sim_p2p.restype = i32
+    L.ccoll_bcast_sim_p2p.argtypes = [vp, vp, sz, i32, sz, f32, u32, vp]
+    L.ccoll_allreduce_sim_p2p.restype = i32
+    L.ccoll_allreduce_sim_p2p.argtypes = [vp, vp, i32, sz, f32, u32, vp, vp]
     L.ccoll_reduce_step_op.restype = i32
     L.ccoll_reduce_step_op.argtypes = [vp, sz, vp, sz, f32, u32, i32, vp, vp, vp, vp]
     L.ccoll_allreduce_sim_op.restype = i32
@@ -166,6 +171,17 @@ def ccoll_bcast_sim(root, out, out_rank_stride, P, eb, mode=BCAST, chunk_bytes=N
                                  _ptr(chunk_bytes), _stream(stream)), "ccoll_bcast_sim")
 
 
+def ccoll_bcast_sim_p2p(root, out, out_rank_stride, P, eb, block_len=BLOCK_LEN, stream=None):
+    _check(lib().ccoll_bcast_sim_p2p(_ptr(root), _ptr(out), out_rank_stride, P, root.numel(), eb, block_len,
+                                     _stream(stream)), "ccoll_bcast_sim_p2p")
+
+
+def ccoll_allreduce_sim_p2p(x, out, eb, bytes_moved=None, block_len=BLOCK_LEN, stream=None):
+    P, n = x.shape
+    _check(lib().ccoll_allreduce_sim_p2p(_ptr(x), _ptr(out), P, n, eb, block_len, _ptr(bytes_moved),
+                                         _stream(stream)), "ccoll_allreduce_sim_p2p")
+
+
 def ccoll_compress_noalloc(x, eb, out, out_bytes, status, block_len=BLOCK_LEN, stream=None):
     """ccoll_compress without a workspace: the scratch is a fixed array inside the library (see ccoll.h).
     `status` is a zeroed uint32/int32 CUDA tensor of one element that receives device-side errors."""
@@ -224,3 +240,22 @@ def bcast_sim(root, P, eb, mode=BCAST, block_len=BLOCK_LEN):
     ccoll_bcast_sim(root, out, stride, P, eb, mode, cb, block_len)
     _check(ccoll_get_status(), "ccoll_bcast_sim (device)")
     return out, cb
+
+
+def bcast_sim_p2p(root, P, eb, block_len=BLOCK_LEN):
+    n = root.numel()
+    ensure_workspace(n, P)
+    out = torch.zeros((P, n), dtype=torch.float32, device=root.device)
+    ccoll_bcast_sim_p2p(root, out, n, P, eb, block_len)
+    _check(ccoll_get_status(), "ccoll_bcast_sim_p2p (device)")
+    return out
+
+
+def allreduce_sim_p2p(x, eb, block_len=BLOCK_LEN):
+    P, n = x.shape
+    ensure_workspace(n, P)
+    out = torch.empty_like(x)
+    moved = torch.zeros(1, dtype=torch.int64, device=x.device)
+    ccoll_allreduce_sim_p2p(x, out, eb, moved, block_len)
+    _check(ccoll_get_status(), "ccoll_allreduce_sim_p2p (device)")
+    return out, int(moved.item())

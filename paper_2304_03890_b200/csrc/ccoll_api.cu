@@ -226,8 +226,8 @@ int ccoll_allreduce_sim(const float* in, float* out, int P, size_t n, float abs_
   return ccoll_allreduce_sim_op(in, out, P, n, abs_err_bound, block_len, CCOLL_SUM, bytes_moved, stream);
 }
 
-int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
-                           int op, uint64_t* bytes_moved, void* stream) {
+static int allreduce_replay(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                            int op, bool p2p, uint64_t* bytes_moved, void* stream) {
   if (P < 1 || (size_t)P > kMaxJobs) return CCOLL_ERR_INVALID_ARG;
   if (op != CCOLL_SUM && op != CCOLL_MAX && op != CCOLL_MIN && op != CCOLL_AVG) return CCOLL_ERR_INVALID_ARG;
   size_t C = ccoll_chunk_len(n, P, block_len);
@@ -268,7 +268,7 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
     b.s_stride = S;
     b.out_cap = S;
     b.moved = bytes_moved;
-    b.moved_mult = (k == P - 1) ? (uint32_t)(P - 1) : 1u;
+    b.moved_mult = (k == P - 1 && !p2p) ? (uint32_t)(P - 1) : 1u;
     b.tiles_per_job = (uint32_t)Gc;
     b.state_stride = state_words((uint32_t)Gc);
     if (k == 0) {
@@ -289,6 +289,48 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
     }
     if ((rc = check_launch()) != CCOLL_OK) return rc;
   }
+  if (p2p) {
+    // CPR-P2P allgather: the stream is decompressed at every hop and compressed again before the next one.
+    // Chunk c's owner is rank c-1, so hop h delivers it to rank c + h - 1.
+    for (int h = 1; h <= P - 1; ++h) {
+      DecodeBatch d;
+      std::memset(&d, 0, sizeof(d));
+      d.sin = buf[cur];
+      d.s_stride = S;
+      d.sin_bytes = bytes[cur];
+      d.out = out;
+      d.out_rank_stride = n;
+      d.chunk_len = C;
+      d.n = n;
+      d.P = P;
+      d.skip_mode = 4;
+      d.rot = h - 1;
+      d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+      if (Gc && !launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s)) return CCOLL_ERR_CUDA;
+      if ((rc = check_launch()) != CCOLL_OK) return rc;
+      if (h == P - 1) break;
+      uint32_t epoch;
+      if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+      EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+      b.x = out;  // what the rank has just received
+      b.x_rank_stride = n;
+      b.chunk_len = C;
+      b.n = n;
+      b.P = P;
+      b.rot = h - 1;
+      b.sout = buf[cur ^ 1];
+      b.s_stride = S;
+      b.out_cap = S;
+      b.out_bytes = bytes[cur ^ 1];
+      b.moved = bytes_moved;
+      b.tiles_per_job = (uint32_t)Gc;
+      b.state_stride = state_words((uint32_t)Gc);
+      if (!launch_compress(b, gx, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
+      if ((rc = check_launch()) != CCOLL_OK) return rc;
+      cur ^= 1;
+    }
+    return CCOLL_OK;
+  }
   // allgather: every rank but the owner decodes the final stream of every chunk
   DecodeBatch d;
   std::memset(&d, 0, sizeof(d));
@@ -304,6 +346,16 @@ int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float a
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
   if (Gc && !launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   return check_launch();
+}
+
+int ccoll_allreduce_sim_op(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                           int op, uint64_t* bytes_moved, void* stream) {
+  return allreduce_replay(in, out, P, n, abs_err_bound, block_len, op, false, bytes_moved, stream);
+}
+
+int ccoll_allreduce_sim_p2p(const float* in, float* out, int P, size_t n, float abs_err_bound, uint32_t block_len,
+                            uint64_t* bytes_moved, void* stream) {
+  return allreduce_replay(in, out, P, n, abs_err_bound, block_len, CCOLL_SUM, true, bytes_moved, stream);
 }
 
 int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float abs_err_bound,
@@ -366,6 +418,69 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
     if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s)) return CCOLL_ERR_CUDA;
   }
   return check_launch();
+}
+
+int ccoll_bcast_sim_p2p(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float abs_err_bound,
+                        uint32_t block_len, void* stream) {
+  if (P < 1 || (size_t)P > kMaxJobs) return CCOLL_ERR_INVALID_ARG;
+  size_t C = ccoll_chunk_len(n, P, block_len);
+  int rc = check_common(C, abs_err_bound, block_len);
+  if (rc != CCOLL_OK) return rc;
+  if (((!root_in || !out) && n) || !aligned16(root_in) || !aligned16(out) || (out_rank_stride % 4) ||
+      (P > 1 && out_rank_stride < n) || root_in == out)
+    return CCOLL_ERR_INVALID_ARG;
+  Workspace* ws;
+  if ((rc = current_ws(&ws)) != CCOLL_OK) return rc;
+  const size_t S = align_up(ccoll_compress_bound(C, block_len), 256);
+  if (P > 1 && ws->bytes < kOffStreams + (size_t)P * S) return CCOLL_ERR_CAPACITY;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (n && cudaMemcpyAsync(out, root_in, 4 * n, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CCOLL_ERR_CUDA;
+  const size_t Gc = groups_of(C);
+  if (P == 1 || Gc == 0) return CCOLL_OK;
+  uint8_t* buf = ws->ptr + kOffStreams;
+  uint64_t* bytes = reinterpret_cast<uint64_t*>(ws->ptr + kOffJobBytes);
+  // Rank r receives from r with its highest set bit cleared, so its copy has been compressed and decompressed
+  // popcount(r) times and ranks of equal depth hold equal data: one compress + decompress per depth (the rank
+  // 2^d - 1 is the first of depth d), then copies to the other ranks of that depth.
+  for (int d = 1; (1 << d) - 1 < P; ++d) {
+    const int first = (1 << d) - 1;
+    const float* src = d == 1 ? root_in : out + (size_t)((1 << (d - 1)) - 1) * out_rank_stride;
+    float* dst = out + (size_t)first * out_rank_stride;
+    uint32_t epoch;
+    if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
+    EncodeBatch b = make_encode(ws, epoch, abs_err_bound);
+    b.x = src;
+    b.chunk_len = C;
+    b.n = n;
+    b.P = P;
+    b.sout = buf;
+    b.s_stride = S;
+    b.out_cap = S;
+    b.out_bytes = bytes;
+    b.tiles_per_job = (uint32_t)Gc;
+    b.state_stride = state_words((uint32_t)Gc);
+    if (!launch_compress(b, (uint32_t)Gc, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
+    if ((rc = check_launch()) != CCOLL_OK) return rc;
+    DecodeBatch dd;
+    std::memset(&dd, 0, sizeof(dd));
+    dd.sin = buf;
+    dd.s_stride = S;
+    dd.sin_bytes = bytes;
+    dd.out = dst;
+    dd.out_rank_stride = out_rank_stride;
+    dd.chunk_len = C;
+    dd.n = n;
+    dd.P = P;
+    dd.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+    if (!launch_decode(dd, (uint32_t)Gc, (uint32_t)P, 1, s)) return CCOLL_ERR_CUDA;
+    if ((rc = check_launch()) != CCOLL_OK) return rc;
+    for (int r = first + 1; r < P; ++r) {
+      if (__builtin_popcount((unsigned)r) != d) continue;
+      if (cudaMemcpyAsync(out + (size_t)r * out_rank_stride, dst, 4 * n, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return CCOLL_ERR_CUDA;
+    }
+  }
+  return CCOLL_OK;
 }
 
 }  // extern "C"

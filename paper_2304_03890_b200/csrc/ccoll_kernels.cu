@@ -1204,7 +1204,8 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   if (g >= jg.G) return;
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
-  float* out = b.scatter ? b.out + (uint64_t)y * b.out_rank_stride : b.out + (uint64_t)z * b.out_rank_stride + jg.lo;
+  const uint32_t dest = b.skip_mode == 4 ? (y + (uint32_t)b.rot) % (uint32_t)b.P : z;
+  float* out = b.scatter ? b.out + (uint64_t)y * b.out_rank_stride : b.out + (uint64_t)dest * b.out_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
   StreamView sv;
   float4 v[8];

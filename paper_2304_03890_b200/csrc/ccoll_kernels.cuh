@@ -80,7 +80,9 @@ struct DecodeBatch {
   uint64_t chunk_len;
   uint64_t n;
   int P;
-  int skip_mode;   // 0 none; 1 skip rank z == (y-1) mod P (the chunk's owner); 2 skip z == 0; 3 skip y == 0
+  int skip_mode;   // 0 none; 1 skip rank z == (y-1) mod P (the chunk's owner); 2 skip z == 0; 3 skip y == 0;
+                   // 4: one destination per chunk, rank (y + rot) mod P (grid.z = 1)
+  int rot;
   int scatter;     // 1: job y writes at out + y*out_rank_stride; 0: at out + z*out_rank_stride + y*C
   uint32_t prefetch_distance;  // groups ahead whose payload a CTA asks L2 for (set by the launcher)
   uint32_t* status;

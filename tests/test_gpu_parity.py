@@ -306,3 +306,27 @@ def test_average_allreduce_matches_oracle(P, n):
     with pytest.raises(B.CcollError) as e:
         B.reduce_step(dev(s0), dev(xs[0]), eb, op=B.AVG)
     assert e.value.code == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("P", [1, 2, 5, 8, 13])
+def test_p2p_bcast_matches_oracle(P):
+    c = fields.config1(n=128 * 70 + 9)
+    x, eb = c["x"].numpy(), float(np.float32(c["eb"]))
+    x = np.ascontiguousarray(x[: x.size // 4 * 4])
+    ref, hops = ccz.bcast_sim_p2p(x, P, eb)
+    got = B.bcast_sim_p2p(dev(x), P, eb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes()
+    if P > 1:   # rank stride shorter than the buffer: the copies would overlap
+        with pytest.raises(B.CcollError) as e:
+            B.ccoll_bcast_sim_p2p(dev(x), torch.empty(P * x.size, device="cuda"), x.size - 4, P, eb)
+        assert e.value.code == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("P,n", [(1, 900), (2, 5000), (4, 128 * 37 + 4), (8, 32 * 32 * 40)])
+def test_p2p_allreduce_matches_oracle(P, n):
+    c = fields.config3(P=max(P, 2), shape=(32, 32, 40), sigma=3.0)
+    xs = np.ascontiguousarray(c["x"].numpy()[:P, :n])
+    eb = float(np.float32(c["eb"]))
+    ref, ref_moved = ccz.allreduce_sim_p2p(xs, eb)
+    got, moved = B.allreduce_sim_p2p(dev(xs), eb)
+    assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
