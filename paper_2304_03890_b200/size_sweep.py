@@ -1,0 +1,75 @@
+"""Message-size sweep with quality figures, shaped like the paper's evaluation (Sec. IV: message sizes of
+278 / 478 / 678 MB, error bounds 1e-2 .. 1e-4 of the range, PSNR and NRMSE of the reconstructed data).
+
+    python -m paper_2304_03890_b200.size_sweep [--sizes-mb 278,478,678] [--rel-eb 1e-2,1e-3,1e-4] [--P 8]
+
+For every size (a smooth 3-D field of that many bytes, the recipe of the 512x512x256 benchmark field) and
+bound it prints the compression ratio, the device time of compress, decompress and the replayed all-reduce
+over P virtual ranks (the buffer viewed as P rank buffers), and PSNR / NRMSE / largest error of the round trip.
+Timing runs through the C ABI; the quality figures are plain reductions over the decoded buffer.
+"""
+import argparse
+import math
+
+import torch
+
+from . import binding as B
+from . import fields
+
+
+def timed(fn, reps=5):
+    fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def quality(x, y):
+    """PSNR (dB, peak = value range), NRMSE (RMSE / value range) and the largest absolute error."""
+    rng = float(x.max() - x.min())
+    d = y.double() - x.double()
+    rmse = math.sqrt(float((d * d).mean()))
+    psnr = float("inf") if rmse == 0 else 20 * math.log10(rng / rmse)
+    return psnr, rmse / rng, float(d.abs().max())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--sizes-mb", default="278,478,678")
+    ap.add_argument("--rel-eb", default="1e-2,1e-3,1e-4")
+    ap.add_argument("--P", type=int, default=8)
+    args = ap.parse_args()
+    P = args.P
+    print("size_MB rel_eb CR compress_ms GB/s decompress_ms GB/s allreduce_ms PSNR_dB NRMSE max_err/eb")
+    for mb in (float(v) for v in args.sizes_mb.split(",")):
+        # 512 x 256 cells per plane; as many planes as the size asks for, a multiple of 4*P values in all
+        planes = max(1, round(mb * 1e6 / 4 / (512 * 256)))
+        x = fields.smooth_field((planes, 512, 256), 8.0, -100.0, 100.0, fields.seed_for(2, int(mb)), "cuda").reshape(-1)
+        n = x.numel() // (4 * P) * (4 * P)
+        x = x[:n].contiguous()
+        B.ensure_workspace(n, P)
+        s = torch.empty(B.ccoll_compress_bound(n), dtype=torch.uint8, device="cuda")
+        nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+        dec = torch.empty_like(x)
+        ar = torch.empty_like(x)
+        for rel in (float(v) for v in args.rel_eb.split(",")):
+            eb = float(fields.eb_from_range(x, rel))
+            t_c = timed(lambda: B.ccoll_compress(x, eb, s, nb))
+            nbytes = int(nb.item())
+            t_d = timed(lambda: B.ccoll_decompress(s, nbytes, n, dec))
+            t_a = timed(lambda: B.ccoll_allreduce_sim(x.view(P, n // P), ar.view(P, n // P), eb), reps=3)
+            assert B.ccoll_get_status() == B.OK
+            psnr, nrmse, emax = quality(x, dec)
+            print(f"{4 * n / 1e6:7.1f} {rel:6.0e} {4 * n / nbytes:5.2f} {t_c:8.3f} {4 * n / t_c / 1e6:6.0f} "
+                  f"{t_d:8.3f} {4 * n / t_d / 1e6:6.0f} {t_a:8.3f} {psnr:7.2f} {nrmse:.2e} {emax / eb:.3f}")
+        del x, s, dec, ar
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()
