@@ -1094,10 +1094,7 @@ __device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
 // ---------------------------------------------------------------------------------------------------
 // kernels
 // ---------------------------------------------------------------------------------------------------
-#ifndef CCOLL_EXP_CTAS
-#define CCOLL_EXP_CTAS 6
-#endif
-__global__ void __launch_bounds__(kThreads, CCOLL_EXP_CTAS) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
+__global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;

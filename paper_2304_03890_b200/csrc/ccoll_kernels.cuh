@@ -23,11 +23,7 @@ constexpr int kThreads = 32 * kWarps;
 constexpr int kHeaderBytes = 32;
 constexpr int kMaxRecord = 5 + kL / 4 + 4 * kL;                       // 549
 constexpr int kMaxGroupBytes = 2 * kGroupBlocks + kGroupBlocks * kMaxRecord;  // 17632 (a multiple of 4)
-#ifdef CCOLL_EXP_IMGWORDS
-constexpr int kImgWords = CCOLL_EXP_IMGWORDS;
-#else
 constexpr int kImgWords = kMaxGroupBytes / 4 + 24;                    // image + slack for 5-word windows
-#endif
 
 // status codes mirrored from ccoll.h
 constexpr uint32_t kErrCapacity = 3, kErrCorrupt = 4, kErrTimeout = 5;
