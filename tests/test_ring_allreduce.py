@@ -1,0 +1,99 @@
+"""The real-rank ring (paper_2304_03890_b200/ring.py): gloo ranks on CPU with a codec built on the oracle check
+the schedule (every rank's result must equal its row of the oracle's replay, bit for bit, and the bytes sent
+must add up to the replay's traffic); on a GPU the same ring runs with the C-ABI codec, its ranks sharing the
+one device (independent kernels, nothing waits on another rank inside a kernel) and gloo carrying the streams."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+class OracleCodec:
+    """CPU stand-in for the device codec: the oracle's compress / reduce step / decompress on torch tensors."""
+
+    def __init__(self, eb, op=0, block_len=128):
+        from oracle import ccz
+        self.ccz, self.eb, self.op, self.block_len = ccz, float(eb), op, block_len
+
+    def empty_stream(self, nbytes, like):
+        return torch.empty(nbytes, dtype=torch.uint8)
+
+    def compress(self, x):
+        return torch.from_numpy(self.ccz.compress(x.numpy(), self.eb).copy())
+
+    def reduce_step(self, stream, local, want_result):
+        if want_result:
+            s, tot = self.ccz.reduce_step(stream.numpy(), local.numpy(), self.eb, want_sum=True, op=self.op)
+            return torch.from_numpy(s.copy()), torch.from_numpy(tot.copy())
+        return torch.from_numpy(self.ccz.reduce_step(stream.numpy(), local.numpy(), self.eb, op=self.op).copy()), None
+
+    def decompress(self, stream, n, out):
+        out.copy_(torch.from_numpy(self.ccz.decompress(stream.numpy(), n).copy()))
+
+
+def _inputs(world, n):
+    from paper_2304_03890_b200 import fields
+    c = fields.config3(P=max(world, 2), shape=(24, 24, 32), sigma=3.0)
+    return np.ascontiguousarray(c["x"].numpy()[:world, :n]), float(np.float32(c["eb"]))
+
+
+def _worker(rank, world, port, n, op, use_gpu, outdir):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2304_03890_b200 import ring
+    xs, eb = _inputs(world, n)
+    if use_gpu:
+        codec = ring.GpuCodec(eb, op)
+        x = torch.from_numpy(xs[rank].copy()).cuda()
+    else:
+        codec = OracleCodec(eb, op)
+        x = torch.from_numpy(xs[rank].copy())
+    out, sent = ring.c_allreduce(x, codec)
+    torch.save({"out": out.cpu(), "sent": sent}, os.path.join(outdir, f"r{rank}.pt"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def _run_and_check(tmp_path, world, n, op, use_gpu):
+    from oracle import ccz
+    port = _free_port()
+    mp.spawn(_worker, args=(world, port, n, op, use_gpu, str(tmp_path)), nprocs=world, join=True)
+    xs, eb = _inputs(world, n)
+    ref, ref_moved = ccz.allreduce_sim(xs, eb, op=op)
+    sent = 0
+    for r in range(world):
+        got = torch.load(os.path.join(str(tmp_path), f"r{r}.pt"))
+        assert got["out"].numpy().tobytes() == ref[r].tobytes(), f"rank {r}"
+        sent += got["sent"]
+    assert sent == ref_moved
+
+
+@pytest.mark.parametrize("world,n", [(2, 5000), (3, 128 * 37 + 5), (4, 24 * 24 * 32)])
+def test_ring_matches_replay_on_cpu_ranks(tmp_path, world, n):
+    _run_and_check(tmp_path, world, n, 0, use_gpu=False)
+
+
+def test_ring_max_on_cpu_ranks(tmp_path):
+    _run_and_check(tmp_path, 3, 4096 * 2 + 77, 1, use_gpu=False)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,n", [(2, 5000), (3, 24 * 24 * 32)])
+def test_ring_with_the_device_codec(tmp_path, world, n):
+    _run_and_check(tmp_path, world, n, 0, use_gpu=True)
