@@ -17,6 +17,10 @@
 // of the group's payload, which leaves as coalesced word stores at the offset a decoupled look-back yields.
 #include "ccoll_kernels.cuh"
 
+#include <cstring>
+
+#include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; nothing links libcuda)
+
 namespace ccoll {
 #ifdef CCOLL_TIMELINE  // development aid: per-CTA phase timestamps (never compiled into the shipped library)
 __device__ unsigned long long g_timeline[8192 * 16];
@@ -158,7 +162,7 @@ struct Smem {
   uint32_t fail;
 };
 constexpr int kCtlBytes = (sizeof(Smem) + 127) / 128 * 128;
-extern __shared__ __align__(128) uint8_t dyn_smem[];
+extern __shared__ __align__(1024) uint8_t dyn_smem[];
 
 // The image is built with atomic ORs, so it must start as zeros.  Only its front (10 KB, more than most
 // groups need) is cleared up front; a group whose payload turns out longer clears the rest once its size is
@@ -230,12 +234,64 @@ __device__ __forceinline__ void pad_ragged(uint8_t* rows, const LaneGeom& lg) {
   }
   __syncwarp();
 }
-// Put the lane's 32 values (held in v) into its slice of the rows.
-__device__ __forceinline__ void write_slice(uint8_t* rows, const float4 (&v)[8]) {
-  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) slice[j] = v[j];
+// ---- tiles moved by the TMA unit -------------------------------------------------------------------
+// A group of 4096 fp32 values is a tile of 128 rows x 128 bytes (row = one lane's slice).  The TMA unit moves
+// such a tile between global and shared memory in one instruction, past the load/store pipe, and applies the
+// 128-byte swizzle on the way: inside every 1024-byte span the 16-byte piece j of row r sits at piece
+// j ^ (r & 7).  A lane that walks its own row piece by piece then meets no bank conflict although the rows
+// are only 128 bytes apart (no padding): byte offset o of lane t's row is at  rows + 128 t + (o ^ 16 (t & 7)),
+// which for offsets below 128 is  (rows + 128 t + 16 (t & 7)) ^ o  — one XOR per access.
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// shared-space address of byte 0 of the calling lane's swizzled row; XOR it with a byte offset < 128
+__device__ __forceinline__ uint32_t swz_row(const uint8_t* rows) {
+  return smem_u32(rows) + 128u * threadIdx.x + 16u * (threadIdx.x & 7u);
 }
+__device__ __forceinline__ void sts128(uint32_t a, const float4& v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+// generic-proxy writes to shared memory must be fenced before the TMA unit (async proxy) reads them
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One thread: store the 128 x 128-byte tile at `rows` to rows [row0, row0+128) of plane `plane` of the tensor,
+// and wait until shared memory has been read (the CTA may then exit or reuse it).
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, const uint8_t* rows, uint32_t row0, uint32_t plane) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
+               "r"(row0), "r"(plane), "r"(smem_u32(rows))
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// Put the lane's 32 values into its swizzled row.
+__device__ __forceinline__ void write_row_swz(uint8_t* rows, const float4 (&v)[8]) {
+  const uint32_t a0 = swz_row(rows);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) sts128(a0 ^ (16u * j), v[j]);
+}
+// Coalesced 128-bit stores from swizzled rows, with bounds: the path of a group that is not complete (and of
+// any group when no tensor map could be made).
+__device__ __forceinline__ void store_rows_swz(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint32_t cnt = group_count(jg, g);
+  float* dst = out + (size_t)g * kGroupValues;
+  const uint32_t base = smem_u32(rows);
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid, row = f >> 3, piece = f & 7u;
+    const float4 t = lds128(base + 128u * row + 16u * (piece ^ (row & 7u)));
+    if (4u * f + 4u <= cnt) {
+      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+    } else {
+      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
+      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
+      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+    }
+  }
+}
+
 // Send the group's values from the rows to global memory with coalesced 128-bit streaming stores (the
 // mirror image of load_rows).  A __syncthreads must separate it from the writes of the slices.
 __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
@@ -1190,7 +1246,8 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
 
 // The incoming image is dead once every lane holds its decoded values in registers, so the rows the values
 // leave through reuse the same shared memory: 18 KB per CTA, which lets 9 CTAs share an SM.
-__global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b) {
+__global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b,
+                                                                   const __grid_constant__ CUtensorMap out_map) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);  // only sm.img is used here
   uint8_t* rows = dyn_smem;                        // aliases sm.img
   const uint32_t g = blockIdx.x, y = blockIdx.y, z = blockIdx.z;
@@ -1224,10 +1281,21 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   }
   TL(3);
   __syncthreads();  // every lane is done reading the image
-  write_slice(rows, v);
-  __syncthreads();
-  TL(4);
-  store_rows(rows, out, jg, g);
+  write_row_swz(rows, v);
+  if (b.use_tma && group_count(jg, g) == (uint32_t)kGroupValues && (smem_u32(rows) & 1023u) == 0u) {
+    // a complete group leaves as one tile: rows [first value / 32, +128) of the destination's plane
+    fence_proxy_async();
+    __syncthreads();
+    TL(4);
+    if (threadIdx.x == 0) {
+      const uint32_t row0 = ((b.scatter ? 0u : jg.lo) + g * (uint32_t)kGroupValues) >> 5;
+      tma_store_tile(&out_map, rows, row0, b.out_rank_stride ? (b.scatter ? y : dest) : 0u);
+    }
+  } else {
+    __syncthreads();
+    TL(4);
+    store_rows_swz(rows, out, jg, g);
+  }
   TL(5);
 }
 
@@ -1241,6 +1309,32 @@ constexpr int kSmemDecode = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRo
 // are resident at a time (the distance of their L2 prefetch).
 bool g_ready[64];
 uint32_t g_slots[64], g_slots_decode[64];
+// Tensor map of a buffer seen as [32 fp32][rows][planes] with 128-byte rows, tile = 32 x 128 x 1, 128-byte
+// swizzle.  The encoder is a driver entry point looked up once through the runtime.  False if it cannot be
+// had or refuses the arguments: the kernels then use their plain load/store paths.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes) {
+  static EncodeTiledFn encode = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      fn = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+  }();
+  if (!encode || (reinterpret_cast<uintptr_t>(base) & 15u)) return false;
+  if (planes > 1 && ((plane_stride_bytes & 15u) || plane_stride_bytes >= (1ull << 40))) return false;
+  const cuuint64_t dims[3] = {32u, rows, planes ? planes : 1u};
+  const cuuint64_t strides[2] = {128u, planes > 1 ? plane_stride_bytes : 128u * rows};
+  const cuuint32_t box[3] = {32u, 128u, 1u};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool device_ready() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
@@ -1295,7 +1389,13 @@ bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint
   DecodeBatch b = b0;
   const uint32_t streams = jobs * ranks;  // CTAs are issued x-fastest over (group, stream, rank)
   b.prefetch_distance = streams == 1 ? g_slots_decode[dev] : (g_slots_decode[dev] + streams - 1) / streams;
-  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b);
+  // The output as a tensor of 128-byte rows: [32 values][rows of a destination][destinations].
+  CUtensorMap map;
+  std::memset(&map, 0, sizeof(map));
+  const uint64_t rows = (b.scatter ? b.chunk_len : b.n) / 32u;
+  const uint64_t planes = b.out_rank_stride ? (b.scatter ? jobs : (b.skip_mode == 4 ? (uint32_t)b.P : ranks)) : 1u;
+  b.use_tma = rows >= 128u && make_tile_map(&map, b.out, rows, planes, b.out_rank_stride * 4u) ? 1 : 0;
+  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b, map);
   return true;
 }
 
