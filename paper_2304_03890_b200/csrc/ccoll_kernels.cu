@@ -38,8 +38,7 @@ __device__ unsigned long long g_timeline[8192 * 16];
 namespace {
 constexpr uint32_t kFull = 0xffffffffu;
 constexpr int kSliceVals = 32;                      // values per lane
-constexpr int kSliceBytes = 144;                    // 128 data bytes + 16 pad
-constexpr int kRowsBytes = kThreads * kSliceBytes;  // 18432
+constexpr int kRowsBytes = kThreads * kSliceVals * 4;  // 16384: one 128-byte row per lane, no padding (swizzled)
 
 // ---------------------------------------------------------------------------------------------------
 // small helpers
@@ -160,8 +159,9 @@ struct Smem {
   uint32_t blk_R[kGroupBlocks];          // 0 = constant or absent block
   uint32_t prefix;                       // exclusive prefix of this group, in words
   uint32_t fail;
+  alignas(8) uint64_t bar;               // mbarrier the TMA load of the rows completes on
 };
-constexpr int kCtlBytes = (sizeof(Smem) + 127) / 128 * 128;
+constexpr int kCtlBytes = (sizeof(Smem) + 1023) / 1024 * 1024;  // the rows behind it need 1024-byte alignment
 extern __shared__ __align__(1024) uint8_t dyn_smem[];
 
 // The image is built with atomic ORs, so it must start as zeros.  Only its front (10 KB, more than most
@@ -180,9 +180,6 @@ __device__ __forceinline__ void zero_image_rest(uint32_t* img) {  // whole CTA; 
   __syncthreads();
 }
 
-// Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
-// (128-bit streaming loads) and scatters them into the padded slices; in round r thread tid moves the
-// float4 number r*128 + tid of the group.  A __syncthreads must follow before the slices are read.
 // Ask L2 for the fp32 values of a group that a later CTA will load (one 128-byte line per thread).  Issued by
 // the CTA that currently occupies the SM slot that later CTA will get, so its loads find the data in L2.
 __device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg, uint32_t g) {
@@ -190,17 +187,107 @@ __device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg
   const uint32_t first = g * (uint32_t)kGroupValues + 32u * threadIdx.x;
   if (first < jg.len) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + first));
 }
-// Bring the group's fp32 values into the rows: every warp reads 512 contiguous bytes per instruction
-// (128-bit streaming loads) and scatters them into the padded slices; in round r thread tid moves the
-// float4 number r*128 + tid of the group.  A __syncthreads must follow before the slices are read.
-// (Letting every lane fetch its own 128 bytes with 256-bit loads needs no transposition and no barrier, but
-// each such load touches 32 lines and the load/store pipe, already the busiest unit here, made it slower.)
-__device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
+
+// ---- rows: the group's values as a tile the TMA unit moves ---------------------------------------------
+// A group of 4096 fp32 values is a tile of 128 rows x 128 bytes, row t = the 32 values of lane t.  The TMA unit
+// moves such a tile between global and shared memory in one instruction, past the load/store pipe, and applies
+// the 128-byte swizzle on the way: inside every 1024-byte span the 16-byte piece j of row r sits at piece
+// j ^ (r & 7).  A lane that walks its own row piece by piece then meets no bank conflict although the rows
+// are only 128 bytes apart (no padding).  Byte offset o < 128 of row t is at  128 t + (o ^ 16 (t & 7))  =
+// (128 t + 16 (t & 7)) ^ o : one XOR per access.
+struct Row {
+  uint8_t* tile;  // the rows buffer (1024-byte aligned)
+  uint32_t off;   // 128 t + 16 (t & 7)
+  __device__ __forceinline__ float4 quad(uint32_t j) const {
+    return *reinterpret_cast<const float4*>(tile + (off ^ (16u * j)));
+  }
+  __device__ __forceinline__ void set_quad(uint32_t j, const float4& v) const {
+    *reinterpret_cast<float4*>(tile + (off ^ (16u * j))) = v;
+  }
+  __device__ __forceinline__ uint4 words4(uint32_t j) const {
+    return *reinterpret_cast<const uint4*>(tile + (off ^ (16u * j)));
+  }
+  __device__ __forceinline__ uint32_t word(uint32_t i) const {
+    return *reinterpret_cast<const uint32_t*>(tile + (off ^ (4u * i)));
+  }
+  __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const {
+    *reinterpret_cast<uint32_t*>(tile + (off ^ (4u * i))) = v;
+  }
+};
+__device__ __forceinline__ Row row_of(uint8_t* rows, uint32_t t) { return Row{rows, 128u * t + 16u * (t & 7u)}; }
+// The other way to keep a lane's walk over its row free of bank conflicts: rows 144 bytes apart, no swizzle, no
+// XOR.  The TMA unit cannot produce it (a tile is dense), so the values are (un)scattered by the lanes.  The
+// encoder alone, whose integer pipe is its busiest unit, is faster this way; where a tile also has to leave
+// again (decoder, fused round) the swizzled rows win.  Same interface as Row.
+constexpr int kPaddedRowBytes = 144;
+constexpr int kPaddedRowsBytes = kThreads * kPaddedRowBytes;  // 18432
+struct PaddedRow {
+  uint8_t* p;
+  __device__ __forceinline__ float4 quad(uint32_t j) const { return *reinterpret_cast<const float4*>(p + 16u * j); }
+  __device__ __forceinline__ uint4 words4(uint32_t j) const { return *reinterpret_cast<const uint4*>(p + 16u * j); }
+  __device__ __forceinline__ uint32_t word(uint32_t i) const { return *reinterpret_cast<const uint32_t*>(p + 4u * i); }
+  __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const { *reinterpret_cast<uint32_t*>(p + 4u * i) = v; }
+};
+template <class RowT>
+__device__ __forceinline__ RowT make_row(uint8_t* rows, uint32_t t);
+template <>
+__device__ __forceinline__ Row make_row<Row>(uint8_t* rows, uint32_t t) { return row_of(rows, t); }
+template <>
+__device__ __forceinline__ PaddedRow make_row<PaddedRow>(uint8_t* rows, uint32_t t) {
+  return PaddedRow{rows + kPaddedRowBytes * t};
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// generic-proxy writes to shared memory must be fenced before the TMA unit (async proxy) reads them
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One thread: arm the barrier and ask the TMA unit for rows [row0, row0+128) of plane `plane` of the tensor.
+__device__ __forceinline__ void tma_load_tile(const CUtensorMap* map, uint8_t* rows, uint64_t* bar, uint32_t row0,
+                                              uint32_t plane) {
+  const uint32_t b = smem_u32(bar);
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  fence_proxy_async();
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(kRowsBytes) : "memory");
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          smem_u32(rows)),
+      "l"(map), "r"(0), "r"(row0), "r"(plane), "r"(b)
+      : "memory");
+}
+// Every thread that will read the rows: wait for the tile (phase 0 of the barrier).  The wait is bounded;
+// false = it gave up (the caller raises a time-out and does not touch the rows).
+__device__ __forceinline__ bool tma_wait_tile(uint64_t* bar) {
+  const uint32_t b = smem_u32(bar);
+  for (uint32_t tries = 0; tries < (1u << 16); ++tries) {
+    uint32_t done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done)
+        : "r"(b)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+// One thread: store the tile to rows [row0, row0+128) of plane `plane` of the tensor, and wait until shared
+// memory has been read (the CTA may then exit or reuse it).
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, const uint8_t* rows, uint32_t row0, uint32_t plane) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
+               "r"(row0), "r"(plane), "r"(smem_u32(rows))
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
+// Padded rows: every warp reads 512 contiguous bytes per instruction (128-bit streaming loads) and scatters
+// them; in round r thread tid moves the float4 number r*128 + tid of the group, piece (tid & 7) of row
+// 16 r + tid / 8.  Zeros past the end of the data.  A __syncthreads must follow before the rows are read.
+__device__ __forceinline__ void load_rows_padded(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
   const uint32_t cnt = group_count(jg, g);
   const float* src = x + (size_t)g * kGroupValues;
-  float4* dst = reinterpret_cast<float4*>(rows + (tid >> 3) * kSliceBytes + 16u * (tid & 7u));
-  constexpr int kRoundStride = (kThreads / 8) * kSliceBytes / 16;  // float4s between a thread's rounds
+  float4* dst = reinterpret_cast<float4*>(rows + (tid >> 3) * kPaddedRowBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kPaddedRowBytes / 16;  // float4s between a thread's rounds
   if (cnt == (uint32_t)kGroupValues) {  // a complete group: no bounds to watch
     float4 t[8];
 #pragma unroll
@@ -223,92 +310,39 @@ __device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const J
     dst[r * kRoundStride] = v;
   }
 }
-// Ragged slices: values past the end of the data are replaced by the block's first value, so that they
-// cannot change min or max.  (The first value of block b is the first value of slice 4b.)  Whole warp.
-__device__ __forceinline__ void pad_ragged(uint8_t* rows, const LaneGeom& lg) {
-  __syncwarp();
-  if (lg.nv < (uint32_t)kSliceVals) {
-    const float f = *reinterpret_cast<const float*>(rows + (threadIdx.x & ~3u) * kSliceBytes);
-    float* x = reinterpret_cast<float*>(rows + threadIdx.x * kSliceBytes);
-    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) x[i] = f;
-  }
-  __syncwarp();
-}
-// ---- tiles moved by the TMA unit -------------------------------------------------------------------
-// A group of 4096 fp32 values is a tile of 128 rows x 128 bytes (row = one lane's slice).  The TMA unit moves
-// such a tile between global and shared memory in one instruction, past the load/store pipe, and applies the
-// 128-byte swizzle on the way: inside every 1024-byte span the 16-byte piece j of row r sits at piece
-// j ^ (r & 7).  A lane that walks its own row piece by piece then meets no bank conflict although the rows
-// are only 128 bytes apart (no padding): byte offset o of lane t's row is at  rows + 128 t + (o ^ 16 (t & 7)),
-// which for offsets below 128 is  (rows + 128 t + 16 (t & 7)) ^ o  — one XOR per access.
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// shared-space address of byte 0 of the calling lane's swizzled row; XOR it with a byte offset < 128
-__device__ __forceinline__ uint32_t swz_row(const uint8_t* rows) {
-  return smem_u32(rows) + 128u * threadIdx.x + 16u * (threadIdx.x & 7u);
-}
-__device__ __forceinline__ void sts128(uint32_t a, const float4& v) {
-  asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ float4 lds128(uint32_t a) {
-  float4 v;
-  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
-  return v;
-}
-// generic-proxy writes to shared memory must be fenced before the TMA unit (async proxy) reads them
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// One thread: store the 128 x 128-byte tile at `rows` to rows [row0, row0+128) of plane `plane` of the tensor,
-// and wait until shared memory has been read (the CTA may then exit or reuse it).
-__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, const uint8_t* rows, uint32_t row0, uint32_t plane) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
-               "r"(row0), "r"(plane), "r"(smem_u32(rows))
-               : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-// Put the lane's 32 values into its swizzled row.
-__device__ __forceinline__ void write_row_swz(uint8_t* rows, const float4 (&v)[8]) {
-  const uint32_t a0 = swz_row(rows);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) sts128(a0 ^ (16u * j), v[j]);
-}
-// Coalesced 128-bit stores from swizzled rows, with bounds: the path of a group that is not complete (and of
-// any group when no tensor map could be made).
-__device__ __forceinline__ void store_rows_swz(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+// The same tile without the TMA unit (a group that is not complete, or no tensor map): coalesced 128-bit
+// loads, bounds watched, zeros past the end; thread tid moves the float4 number r*128 + tid in round r, which
+// is piece (tid & 7) of row 16 r + tid / 8.  A __syncthreads must follow before the rows are read.
+__device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
   const uint32_t cnt = group_count(jg, g);
-  float* dst = out + (size_t)g * kGroupValues;
-  const uint32_t base = smem_u32(rows);
+  const float* src = x + (size_t)g * kGroupValues;
+  uint8_t* dst = rows + 128u * (tid >> 3) + 16u * ((tid & 7u) ^ ((tid >> 3) & 7u));
 #pragma unroll 1
   for (int r = 0; r < 8; ++r) {
-    const uint32_t f = (uint32_t)r * kThreads + tid, row = f >> 3, piece = f & 7u;
-    const float4 t = lds128(base + 128u * row + 16u * (piece ^ (row & 7u)));
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (4u * f + 4u <= cnt) {
-      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
     } else {
-      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
-      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
-      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
     }
+    *reinterpret_cast<float4*>(dst + 2048 * r) = v;
   }
 }
-
-// Send the group's values from the rows to global memory with coalesced 128-bit streaming stores (the
-// mirror image of load_rows).  A __syncthreads must separate it from the writes of the slices.
+// ... and out: coalesced 128-bit streaming stores from the rows, bounds watched.  A __syncthreads must
+// separate it from the writes of the rows.
 __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
   const uint32_t cnt = group_count(jg, g);
   float* dst = out + (size_t)g * kGroupValues;
-  const float4* src = reinterpret_cast<const float4*>(rows + (tid >> 3) * kSliceBytes + 16u * (tid & 7u));
-  constexpr int kRoundStride = (kThreads / 8) * kSliceBytes / 16;
-  if (cnt == (uint32_t)kGroupValues) {
-#pragma unroll
-    for (int r = 0; r < 8; ++r) __stcs(reinterpret_cast<float4*>(dst) + r * kThreads + tid, src[r * kRoundStride]);
-    return;
-  }
+  const uint8_t* src = rows + 128u * (tid >> 3) + 16u * ((tid & 7u) ^ ((tid >> 3) & 7u));
 #pragma unroll 1
   for (int r = 0; r < 8; ++r) {
     const uint32_t f = (uint32_t)r * kThreads + tid;
-    const float4 t = src[r * kRoundStride];
+    const float4 t = *reinterpret_cast<const float4*>(src + 2048 * r);
     if (4u * f + 4u <= cnt) {
       __stcs(reinterpret_cast<float4*>(dst) + f, t);
     } else {
@@ -317,6 +351,18 @@ __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, cons
       if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
     }
   }
+}
+// Ragged rows: values past the end of the data are replaced by the block's first value, so that they
+// cannot change min or max.  (The first value of block b is the first value of row 4b.)  Whole warp.
+template <class RowT>
+__device__ __forceinline__ void pad_ragged(uint8_t* rows, const LaneGeom& lg) {
+  __syncwarp();
+  if (lg.nv < (uint32_t)kSliceVals) {
+    const uint32_t f = make_row<RowT>(rows, threadIdx.x & ~3u).word(0);
+    const RowT row = make_row<RowT>(rows, threadIdx.x);
+    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) row.set_word(i, f);
+  }
+  __syncwarp();
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -334,13 +380,14 @@ struct Plan {
 
 // Largest and smallest of the lane's 32 values (a NaN wins both), read from the lane's slice.  The loop is
 // unrolled only twice: fully unrolled on register arrays the fused kernel outgrew the 32 KB instruction cache.
-__device__ __forceinline__ void lane_minmax(const float4* x4, float& mx, float& mn) {
-  float4 q = x4[0];
+template <class RowT>
+__device__ __forceinline__ void lane_minmax(const RowT& row, float& mx, float& mn) {
+  float4 q = row.quad(0);
   mx = max3_nan(max_nan(q.x, q.y), q.z, q.w);
   mn = min3_nan(min_nan(q.x, q.y), q.z, q.w);
 #pragma unroll 2
   for (int j = 1; j < 8; ++j) {
-    q = x4[j];
+    q = row.quad(j);
     mx = max3_nan(max3_nan(mx, q.x, q.y), q.z, q.w);
     mn = min3_nan(min3_nan(mn, q.x, q.y), q.z, q.w);
   }
@@ -381,77 +428,26 @@ __device__ __forceinline__ uint32_t code_of(float x, const Plan& p) {
   return __float_as_uint(p.lossless ? x : __fsub_rn(x, p.mu)) >> p.sh;
 }
 
-// Rules R7-R8 for one quad of values with codes q0..q3 (prev = code before q0).  sa_e = 32 - 8*(stored
-// bytes of value e) is taken straight from the leading-zero count of (code xor predecessor): a value
-// stores its significant bytes; `fix` forces at least one stored byte when the field is 4 bytes wide
-// (lead is capped at 3).  Appends the quad's bytes to the lane's staging words and returns the new state.
-struct Stage {
-  uint32_t* wp;     // next staging word
-  uint32_t pendb;   // bits (0, 8, 16, 24) waiting in carry
-  uint32_t carry;   // the partial word, zero above pendb
-  uint32_t Tb;      // bits staged so far
-};
-__device__ __forceinline__ void append_quad(Stage& st, uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3,
-                                            uint32_t sa0, uint32_t sa1, uint32_t sa2, uint32_t sa3) {
-  // the stored (low) bytes of each code, most significant first, as little-endian integers ...
-  const uint32_t e0 = __funnelshift_rc(__byte_perm(q0, 0u, 0x0123), 0u, sa0);
-  const uint32_t e1 = __funnelshift_rc(__byte_perm(q1, 0u, 0x0123), 0u, sa1);
-  const uint32_t e2 = __funnelshift_rc(__byte_perm(q2, 0u, 0x0123), 0u, sa2);
-  const uint32_t e3 = __funnelshift_rc(__byte_perm(q3, 0u, 0x0123), 0u, sa3);
-  // ... concatenated into one 16-byte little-endian string W0..W3
-  const uint32_t s0 = 32u - sa0, s2 = 32u - sa2;
-  const uint32_t lo01 = e0 | __funnelshift_lc(0u, e1, s0), hi01 = __funnelshift_lc(e1, 0u, s0);
-  const uint32_t lo23 = e2 | __funnelshift_lc(0u, e3, s2), hi23 = __funnelshift_lc(e3, 0u, s2);
-  const uint32_t s01 = 64u - sa0 - sa1;  // bits of the first pair, 0..64
-  const bool upper = s01 >= 32u;
-  const uint32_t a = upper ? s01 - 32u : s01;
-  const uint32_t t0 = __funnelshift_lc(0u, lo23, a), t1 = __funnelshift_lc(lo23, hi23, a),
-                 t2 = __funnelshift_lc(hi23, 0u, a);
-  const uint32_t W0 = upper ? lo01 : (lo01 | t0);
-  const uint32_t W1 = upper ? (hi01 | t0) : (hi01 | t1);
-  const uint32_t W2 = upper ? t1 : t2;
-  const uint32_t W3 = upper ? t2 : 0u;
-  // append behind the bits waiting in carry; words past the end are overwritten by the next quad
-  const uint32_t z = st.pendb;
-  const uint32_t V0 = (W0 << z) | st.carry;
-  const uint32_t V1 = __funnelshift_l(W0, W1, z);
-  const uint32_t V2 = __funnelshift_l(W1, W2, z);
-  const uint32_t V3 = __funnelshift_l(W2, W3, z);
-  const uint32_t V4 = __funnelshift_l(W3, 0u, z);
-  st.wp[0] = V0;
-  st.wp[1] = V1;
-  st.wp[2] = V2;
-  st.wp[3] = V3;
-  const uint32_t T4b = 128u - sa0 - sa1 - sa2 - sa3;
-  const uint32_t totb = z + T4b;  // 0..152
-  const uint32_t c01 = (totb & 32u) ? V1 : V0, c23 = (totb & 32u) ? V3 : V2;
-  st.carry = (totb & 128u) ? V4 : ((totb & 64u) ? c23 : c01);
-  st.wp += totb >> 5;
-  st.pendb = totb & 31u;
-  st.Tb += T4b;
-}
-__device__ __forceinline__ void finish_stage(Stage& st) {
-  st.wp[0] = st.carry;  // the last partial word, zero padded
-  st.wp[1] = 0u;        // and a zero word behind it for the realigning copy
-}
-
-// Fast path: all 32 values valid, block not lossless.  The lane's byte string is built in a 64-bit big-endian
-// accumulator (hi:lo, its low `pend` bits waiting to be written): a value's stored bytes are its low
+// Rules R7-R8 for the lane's 32 values.  The lane's byte string is built in a 64-bit big-endian accumulator
+// (hi:lo; Tb = bits appended so far, the low Tb & 31 of them still waiting): a value's stored bytes are its low
 // n = 8 * (stored bytes) bits, appended with two funnel shifts; whenever 32 bits are complete they leave as
 // one word (byte-reversed, since the first byte of the stream is the most significant one).  n comes
 // straight from the leading-zero count of (code xor predecessor); `fix` forces at least one stored byte when
-// the field is 4 bytes wide (lead is capped at 3).  Values are read from the slice quad by quad and the
-// staged words overwrite the slice in place, which is safe because at most 16 bytes are staged per quad and
+// the field is 4 bytes wide (lead is capped at 3).  Values are read from the lane's row quad by quad and the
+// staged words overwrite the row in place, which is safe because at most 16 bytes are staged per quad and
 // quad j is read before anything is written at or behind its position.
-__device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const Plan& p, uint32_t prev, uint32_t& T_out,
-                                               uint32_t& code_lo, uint32_t& code_hi) {
-  const uint32_t fix = (p.B == 4u) ? 1u : 0u;
-  const uint32_t cadj = (4u - p.B) * (85u << 24);
-  const float mu = p.mu;
-  const uint32_t sh = p.sh;
-  uint32_t lo = 0u, hi = 0u, Tb = 0u;  // Tb = bits appended so far; the low (Tb & 31) bits of hi:lo are waiting
+// kGeneral = false: all 32 values valid, block not lossless (loop unrolled twice).  kGeneral = true: ragged
+// rows (values past nv store nothing and have lead code 0) and lossless blocks, rolled.
+template <bool kGeneral, class RowT>
+__device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
+                                          uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  const bool lossless = kGeneral && R == 32u;
+  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
+  const uint32_t fix = (B == 4u) ? 1u : 0u;
+  const uint32_t unused = 4u - B;  // top bytes of the 32-bit code that the field does not have
+  const float mu = __uint_as_float(mu_bits);
+  uint32_t lo = 0u, hi = 0u, Tb = 0u;
   uint32_t clo = 0u, chi = 0u;
-  const float4* x4 = reinterpret_cast<const float4*>(slice);
   auto put = [&](uint32_t q, uint32_t sa) {
     const uint32_t n = 32u - sa;
     const uint32_t t = __funnelshift_lc(0u, q, sa);  // the stored bits, at the top of the word
@@ -459,50 +455,12 @@ __device__ __forceinline__ void emit_lane_fast(uint32_t* slice, const Plan& p, u
     hi = __funnelshift_lc(lo, hi, n);
     lo = __funnelshift_lc(t, lo, n);
     if ((Tn ^ Tb) & 32u)  // a word boundary was crossed (n <= 32: at most one)
-      slice[(Tn >> 5) - 1u] = __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123);
+      row.set_word((Tn >> 5) - 1u, __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123));
     Tb = Tn;
   };
-#pragma unroll 2
+#pragma unroll(kGeneral ? 1 : 2)
   for (int j = 0; j < 8; ++j) {
-    const float4 x = x4[j];
-    const uint32_t q0 = __float_as_uint(__fsub_rn(x.x, mu)) >> sh, q1 = __float_as_uint(__fsub_rn(x.y, mu)) >> sh,
-                   q2 = __float_as_uint(__fsub_rn(x.z, mu)) >> sh, q3 = __float_as_uint(__fsub_rn(x.w, mu)) >> sh;
-    const uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
-                   sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
-    prev = q3;
-    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field; the
-    // quad's four codes enter the 64-bit code string from the top, so that after eight quads quad 0 is lowest
-    const uint32_t cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) << 21) - cadj;
-    clo = __funnelshift_r(clo, chi, 8u);
-    chi = (chi >> 8) | cb;
-    put(q0, sa0);
-    put(q1, sa1);
-    put(q2, sa2);
-    put(q3, sa3);
-  }
-  const uint32_t pend = Tb & 31u;
-  uint32_t* wp = slice + (Tb >> 5);
-  wp[0] = pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u;  // the last partial word, zero padded
-  wp[1] = 0u;                                                        // and a zero word for the realigning copy
-  T_out = Tb >> 3;
-  code_lo = clo;
-  code_hi = chi;
-}
-
-// General path (ragged slices, lossless blocks): rolled loop over the quads, values re-read from the slice.
-// Staging in place is safe: quad j is read before anything is written at or behind its position.
-__device__ __noinline__ void emit_lane_slow(uint32_t* slice, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
-                                            uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
-  const bool lossless = R == 32u;
-  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
-  const uint32_t fix = (B == 4u) ? 1u : 0u;
-  const float mu = __uint_as_float(mu_bits);
-  Stage st = {slice, 0u, 0u, 0u};
-  uint64_t codes = 0ull;
-  const float4* src = reinterpret_cast<const float4*>(slice);
-#pragma unroll 1
-  for (uint32_t j = 0; j < 8u; ++j) {
-    const float4 x = src[j];
+    const float4 x = row.quad(j);
     const uint32_t q0 = __float_as_uint(lossless ? x.x : __fsub_rn(x.x, mu)) >> sh,
                    q1 = __float_as_uint(lossless ? x.y : __fsub_rn(x.y, mu)) >> sh,
                    q2 = __float_as_uint(lossless ? x.z : __fsub_rn(x.z, mu)) >> sh,
@@ -510,35 +468,59 @@ __device__ __noinline__ void emit_lane_slow(uint32_t* slice, uint32_t R, uint32_
     uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
              sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
     prev = q3;
-    uint32_t l0 = (sa0 >> 3) - (4u - B), l1 = (sa1 >> 3) - (4u - B), l2 = (sa2 >> 3) - (4u - B), l3 = (sa3 >> 3) - (4u - B);
-    if (4u * j + 0u >= nv) sa0 = 32u, l0 = 0u;  // values past the end store nothing and have code 0
-    if (4u * j + 1u >= nv) sa1 = 32u, l1 = 0u;
-    if (4u * j + 2u >= nv) sa2 = 32u, l2 = 0u;
-    if (4u * j + 3u >= nv) sa3 = 32u, l3 = 0u;
-    codes |= (uint64_t)(l0 | (l1 << 2) | (l2 << 4) | (l3 << 6)) << (8u * j);
-    append_quad(st, q0, q1, q2, q3, sa0, sa1, sa2, sa3);
+    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field; the
+    // quad's four codes enter the 64-bit code string from the top, so that after eight quads quad 0 is lowest
+    uint32_t cb;
+    if (kGeneral) {
+      uint32_t l0 = (sa0 >> 3) - unused, l1 = (sa1 >> 3) - unused, l2 = (sa2 >> 3) - unused, l3 = (sa3 >> 3) - unused;
+      if (4u * j + 0u >= nv) sa0 = 32u, l0 = 0u;
+      if (4u * j + 1u >= nv) sa1 = 32u, l1 = 0u;
+      if (4u * j + 2u >= nv) sa2 = 32u, l2 = 0u;
+      if (4u * j + 3u >= nv) sa3 = 32u, l3 = 0u;
+      cb = (l0 | (l1 << 2) | (l2 << 4) | (l3 << 6)) << 24;
+    } else {
+      cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) << 21) - unused * (85u << 24);
+    }
+    clo = __funnelshift_r(clo, chi, 8u);
+    chi = (chi >> 8) | cb;
+    put(q0, sa0);
+    put(q1, sa1);
+    put(q2, sa2);
+    put(q3, sa3);
   }
-  finish_stage(st);
-  T_out = st.Tb >> 3;
-  code_lo = (uint32_t)codes;
-  code_hi = (uint32_t)(codes >> 32);
+  const uint32_t pend = Tb & 31u, w = Tb >> 5;
+  // the last partial word, zero padded, and a zero word behind it for the realigning copy — as far as the row
+  // reaches (a row that is full to its last byte has neither; copy_staged reads zeros past the row's end)
+  if (w < 32u) row.set_word(w, pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u);
+  if (w + 1u < 32u) row.set_word(w + 1u, 0u);
+  T_out = Tb >> 3;
+  code_lo = clo;
+  code_hi = chi;
+}
+template <class RowT>
+__device__ __noinline__ void emit_lane_general(RowT row, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
+                                               uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  emit_lane<true, RowT>(row, R, mu_bits, nv, prev, T_out, code_lo, code_hi);
 }
 
-// Copy the lane's T staged bytes from its slice to byte offset dst of the image.  The first and last image
+// Copy the lane's T staged bytes from its row to byte offset dst of the image.  The first and last image
 // word may be shared with a neighbour and are ORed in; the words between are plain stores.
-__device__ __forceinline__ void copy_staged(uint32_t* img, const uint32_t* slice, uint32_t dst, uint32_t T) {
+template <class RowT>
+__device__ __forceinline__ void copy_staged(uint32_t* img, const RowT& row, uint32_t dst, uint32_t T) {
   if (T == 0u) return;
   const uint32_t z = 8u * (dst & 3u);
   uint32_t* out = img + (dst >> 2);
-  const uint32_t nw = ((dst & 3u) + T + 3u) >> 2;  // image words touched
-  atomicOr(&out[0], slice[0] << z);
-  if (nw > 1u) atomicOr(&out[nw - 1u], __funnelshift_l(slice[nw - 2u], slice[nw - 1u], z));
+  const uint32_t nw = ((dst & 3u) + T + 3u) >> 2;  // image words touched, <= 33
+  atomicOr(&out[0], row.word(0) << z);
+  if (nw > 1u) {
+    const uint32_t last = nw - 1u < 32u ? row.word(nw - 1u) : 0u;  // nothing is staged past the row's 32 words
+    atomicOr(&out[nw - 1u], __funnelshift_l(row.word(nw - 2u), last, z));
+  }
   if (nw <= 2u) return;
   const uint32_t ni = nw - 2u;  // interior words 1 .. nw-2
-  const uint4* src = reinterpret_cast<const uint4*>(slice);
   uint32_t prevw = 0u;
   for (uint32_t c = 0; 4u * c <= ni; ++c) {
-    const uint4 cur = src[c];
+    const uint4 cur = row.words4(c);
     const uint32_t w0 = __funnelshift_l(prevw, cur.x, z), w1 = __funnelshift_l(cur.x, cur.y, z),
                    w2 = __funnelshift_l(cur.y, cur.z, z), w3 = __funnelshift_l(cur.z, cur.w, z);
     prevw = cur.w;
@@ -645,21 +627,22 @@ __device__ __forceinline__ void prefix_earlier_super_tiles(Smem& sm, const SizeW
 // Encode the group whose values wait in the lanes' slices (ragged slices already padded; mx, mn = largest and
 // smallest value of the lane's slice): build the payload image, find its place in the stream and copy it
 // out.  The image must have been zeroed (that is made visible by the barrier inside) before the call.
+template <class RowT>
 __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const LaneGeom& lg, const EncodeBatch& b,
                                              const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout, float mx,
                                              float mn, bool tail) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  uint32_t* slice = reinterpret_cast<uint32_t*>(rows + tid * kSliceBytes);
+  const RowT row = make_row<RowT>(rows, tid);
   Plan p = plan_block(mx, mn, lg, b.eb, b.eb_exp);
   // code of the value just before this lane's first one (0 at the start of a block)
-  uint32_t prev = __shfl_up_sync(kFull, code_of(reinterpret_cast<const float*>(slice)[kSliceVals - 1], p), 1);
+  uint32_t prev = __shfl_up_sync(kFull, code_of(__uint_as_float(row.word(kSliceVals - 1)), p), 1);
   if (lg.t == 0u) prev = 0u;
   uint32_t T = 0u, code_lo = 0u, code_hi = 0u;
   if (p.R != 0u) {
     if (tail || p.lossless)
-      emit_lane_slow(slice, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
+      emit_lane_general(row, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
     else
-      emit_lane_fast(slice, p, prev, T, code_lo, code_hi);
+      emit_lane<false, RowT>(row, p.R, p.mu_bits, (uint32_t)kSliceVals, prev, T, code_lo, code_hi);
   }
   uint32_t total;
   const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
@@ -700,7 +683,7 @@ __device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const Lane
     }
     if (p.R) {
       if (8u * lg.t < cbytes) or_u64(sm.img, boff + 5u + 8u * lg.t, code_lo, code_hi);
-      copy_staged(sm.img, slice, boff + 5u + cbytes + excl, T);
+      copy_staged(sm.img, row, boff + 5u + cbytes + excl, T);
     }
   }
 
@@ -922,7 +905,7 @@ __device__ __forceinline__ float reduce_op(float a, float b, int op, float divis
 // the loops are then unrolled only twice, which keeps the fused kernel inside the instruction cache.
 template <bool kToSlice, bool kDivide = false>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8], float4* slice4, int op, float divisor, float& mx,
+                                             float4 (&v)[8], const Row& row, int op, float divisor, float& mx,
                                              float& mn) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
@@ -1039,10 +1022,10 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
   constexpr int kUnroll = kToSlice ? 2 : 8;
   auto put = [&](int j, const float4& r) {
     if (kToSlice) {
-      const float4 a = slice4[j];
+      const float4 a = row.quad(j);
       const float4 o = make_float4(reduce_op<kDivide>(r.x, a.x, op, divisor), reduce_op<kDivide>(r.y, a.y, op, divisor),
                                    reduce_op<kDivide>(r.z, a.z, op, divisor), reduce_op<kDivide>(r.w, a.w, op, divisor));
-      slice4[j] = o;
+      row.set_quad(j, o);
       mx = max3_nan(max3_nan(mx, o.x, o.y), o.z, o.w);  // the encoder's min/max, while the values are at hand
       mn = min3_nan(min3_nan(mn, o.x, o.y), o.z, o.w);
     } else {
@@ -1150,6 +1133,16 @@ __device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
 // ---------------------------------------------------------------------------------------------------
 // kernels
 // ---------------------------------------------------------------------------------------------------
+// A group that cannot be encoded (corrupt input, a wait that ran out): report it, and publish poisoned size
+// words so that no later group waits for this one.
+__device__ __forceinline__ void give_up(const EncodeBatch& b, const JobGeom& jg, uint32_t g, uint32_t y, uint32_t code) {
+  if (threadIdx.x != 0) return;
+  raise(b.status, code);
+  const SizeWords sw = size_words(b, y);
+  st_relaxed_u64(&sw.A[g], pack_state(b.epoch, kFlagPoison, 0));
+  if ((g & 31u) == 31u || g == jg.G - 1u) st_relaxed_u64(&sw.SA[g >> 5], pack_state(b.epoch, kFlagPoison, 0));
+}
+
 __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __grid_constant__ EncodeBatch b) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
@@ -1165,19 +1158,21 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __gri
   const float* x = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
-  load_rows(rows, x, jg, g);
+  load_rows_padded(rows, x, jg, g);
   prefetch_group(x, jg, g + b.prefetch_distance);
   zero_image(sm.img);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
   __syncthreads();
-  if (tail) pad_ragged(rows, lg);
+  if (tail) pad_ragged<PaddedRow>(rows, lg);
   float mx, mn;
-  lane_minmax(reinterpret_cast<const float4*>(rows + threadIdx.x * kSliceBytes), mx, mn);
-  encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
+  lane_minmax(make_row<PaddedRow>(rows, threadIdx.x), mx, mn);
+  encode_group<PaddedRow>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
 }
 
 template <bool kDivide>
-__global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b) {
+__global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_constant__ EncodeBatch b,
+                                                                   const __grid_constant__ CUtensorMap x_map,
+                                                                   const __grid_constant__ CUtensorMap sum_map) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
@@ -1193,8 +1188,15 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const LaneGeom lg = lane_geom(jg, g);
   TL(0);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
-  float4* slice = reinterpret_cast<float4*>(rows + threadIdx.x * kSliceBytes);
-  load_rows(rows, local, jg, g);
+  const Row row = row_of(rows, threadIdx.x);
+  const bool whole = group_count(jg, g) == (uint32_t)kGroupValues && (smem_u32(rows) & 1023u) == 0u;
+  const bool tma = b.use_tma_in && whole;
+  const uint32_t row0 = (jg.lo + g * (uint32_t)kGroupValues) >> 5;  // the group's first row in the rank buffer
+  if (tma) {
+    if (threadIdx.x == 0) tma_load_tile(&x_map, rows, &sm.bar, row0, b.x_rank_stride ? rank : 0u);
+  } else {
+    load_rows(rows, local, jg, g);
+  }
   prefetch_group(local, jg, g + b.prefetch_distance);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
 
@@ -1212,40 +1214,45 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   if (ok) {
     stage_payload(sm, sv);
     prefetch_payload(sv, nxt_a, nxt_e);
-    __syncthreads();  // the image and the local values in the rows are complete
+    __syncthreads();  // the image is complete (and the barrier the tile lands on is initialised)
     TL(1);
-    // decoded + local, one rounded add per value, left in the lane's slice
-    ok = decode_group<true, kDivide>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, slice,
+    if (tma && !tma_wait_tile(&sm.bar)) {
+      give_up(b, jg, g, y, kErrTimeout);
+      return;
+    }
+    // decoded (op) local, one rounded operation per value, left in the lane's row
+    ok = decode_group<true, kDivide>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, row,
                                      b.op, b.divisor, mx, mn);
   }
   TL(2);
-  if (!ok) {
-    // a corrupt input: report it, and keep the look-back chain alive with a poisoned entry
-    if (threadIdx.x == 0) {
-      raise(b.status, kErrCorrupt);
-      const SizeWords sw = size_words(b, y);
-      st_relaxed_u64(&sw.A[g], pack_state(b.epoch, kFlagPoison, 0));
-      if ((g & 31u) == 31u || g == jg.G - 1u) st_relaxed_u64(&sw.SA[g >> 5], pack_state(b.epoch, kFlagPoison, 0));
-    }
+  if (!ok) {  // a corrupt input
+    if (tma && threadIdx.x == 0) tma_wait_tile(&sm.bar);  // the tile in flight must land before the CTA's memory goes
+    give_up(b, jg, g, y, kErrCorrupt);
     return;
   }
-  __syncthreads();  // every thread is done reading the incoming image (and has written its sums)
+  const bool tma_sum = b.sum_out && b.use_tma_sum && whole;
+  if (tma_sum) fence_proxy_async();  // the results just written are about to be read by the TMA unit
+  __syncthreads();  // every thread is done reading the incoming image (and has written its results)
   zero_image(sm.img);
   if (b.sum_out) {
-    store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
-    __syncthreads();  // the slices are about to be reused for staging
+    if (tma_sum) {
+      if (threadIdx.x == 0) tma_store_tile(&sum_map, rows, row0, b.sum_rank_stride ? rank : 0u);
+    } else {
+      store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
+    }
+    __syncthreads();  // the rows are about to be reused for staging
   }
   TL(3);
   if (tail) {
-    pad_ragged(rows, lg);
-    lane_minmax(slice, mx, mn);
+    pad_ragged<Row>(rows, lg);
+    lane_minmax(row, mx, mn);
   }
-  encode_group(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
+  encode_group<Row>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
   TL(7);
 }
 
 // The incoming image is dead once every lane holds its decoded values in registers, so the rows the values
-// leave through reuse the same shared memory: 18 KB per CTA, which lets 9 CTAs share an SM.
+// leave through reuse the same shared memory: 18 KB per CTA (registers then limit an SM to 9 CTAs).
 __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_constant__ DecodeBatch b,
                                                                    const __grid_constant__ CUtensorMap out_map) {
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);  // only sm.img is used here
@@ -1273,7 +1280,8 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
     __syncthreads();
     TL(2);
     float mx_unused, mn_unused;
-    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, nullptr, 0, 0.0f, mx_unused, mn_unused);
+    ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, Row{nullptr, 0u}, 0,
+                             0.0f, mx_unused, mn_unused);
   }
   if (!ok) {
     if (threadIdx.x == 0) raise(b.status, kErrCorrupt);
@@ -1281,7 +1289,11 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   }
   TL(3);
   __syncthreads();  // every lane is done reading the image
-  write_row_swz(rows, v);
+  {
+    const Row row = row_of(rows, threadIdx.x);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) row.set_quad(j, v[j]);
+  }
   if (b.use_tma && group_count(jg, g) == (uint32_t)kGroupValues && (smem_u32(rows) & 1023u) == 0u) {
     // a complete group leaves as one tile: rows [first value / 32, +128) of the destination's plane
     fence_proxy_async();
@@ -1294,7 +1306,7 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   } else {
     __syncthreads();
     TL(4);
-    store_rows_swz(rows, out, jg, g);
+    store_rows(rows, out, jg, g);
   }
   TL(5);
 }
@@ -1302,7 +1314,8 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
 }  // namespace
 
 namespace {
-constexpr int kSmemBytes = kCtlBytes + kRowsBytes;
+constexpr int kSmemBytes = kCtlBytes + kRowsBytes;            // fused round: control block + swizzled rows
+constexpr int kSmemCompress = kCtlBytes + kPaddedRowsBytes;  // encoder: control block + padded rows
 constexpr int kSmemDecode = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
 
 // Per device: opt in to the dynamic shared-memory size once, and learn how many CTAs of the encoding kernels
@@ -1340,12 +1353,12 @@ bool device_ready() {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
   if (!g_ready[dev]) {
     int sms = 0, per_sm = 0;
-    if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ccoll_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCompress) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_reduce_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_reduce_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(ccoll_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDecode) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_compress_kernel, kThreads, kSmemBytes) != cudaSuccess)
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_compress_kernel, kThreads, kSmemCompress) != cudaSuccess)
       return false;
     g_slots[dev] = (uint32_t)(sms * (per_sm > 0 ? per_sm : 1));
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_decode_kernel, kThreads, kSmemDecode) != cudaSuccess)
@@ -1367,19 +1380,27 @@ static EncodeBatch with_prefetch(const EncodeBatch& b, uint32_t jobs) {
   c.prefetch_distance = jobs == 1 ? g_slots[dev] : (g_slots[dev] + jobs - 1) / jobs;
   return c;
 }
+// The fp32 side of an encode batch as a tensor of 128-byte rows: [32 values][rows of a rank][ranks].
+static bool rank_buffer_map(CUtensorMap* map, const float* base, uint64_t n, uint64_t rank_stride, int P) {
+  std::memset(map, 0, sizeof(*map));
+  return base && n / 32u >= 128u && make_tile_map(map, base, n / 32u, rank_stride ? (uint64_t)P : 1u, rank_stride * 4u);
+}
 bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
   const EncodeBatch b = with_prefetch(b0, jobs);
-  ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+  ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemCompress, s>>>(b);
   return true;
 }
 bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
-  const EncodeBatch b = with_prefetch(b0, jobs);
+  EncodeBatch b = with_prefetch(b0, jobs);
+  CUtensorMap x_map, sum_map;
+  b.use_tma_in = rank_buffer_map(&x_map, b.x, b.n, b.x_rank_stride, b.P) ? 1 : 0;
+  b.use_tma_sum = rank_buffer_map(&sum_map, b.sum_out, b.n, b.sum_rank_stride, b.P) ? 1 : 0;
   if (b.op == 3)
-    ccoll_reduce_kernel<true><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+    ccoll_reduce_kernel<true><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b, x_map, sum_map);
   else
-    ccoll_reduce_kernel<false><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b);
+    ccoll_reduce_kernel<false><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b, x_map, sum_map);
   return true;
 }
 bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {

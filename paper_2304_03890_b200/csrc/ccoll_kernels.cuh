@@ -60,6 +60,7 @@ struct EncodeBatch {
   uint32_t state_stride;
   uint32_t epoch;
   uint32_t prefetch_distance;  // groups ahead whose values a CTA asks L2 for (set by the launcher)
+  int use_tma_in, use_tma_sum;  // complete groups of x / sum_out move as TMA tiles (set by the launcher)
   uint32_t* status;         // sticky error word
   float eb;
   int eb_exp;               // biased exponent field of eb
