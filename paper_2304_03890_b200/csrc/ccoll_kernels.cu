@@ -160,9 +160,12 @@ struct Smem {
   uint32_t prefix;                       // exclusive prefix of this group, in words
   uint32_t fail;
   alignas(8) uint64_t bar;               // mbarrier the TMA load of the rows completes on
+  uint64_t bar_in;                       // mbarrier the bulk copy of the incoming payload completes on
 };
 constexpr int kCtlBytes = (sizeof(Smem) + 1023) / 1024 * 1024;  // the rows behind it need 1024-byte alignment
 extern __shared__ __align__(1024) uint8_t dyn_smem[];
+// decode kernel: image (aliased by the output rows) at offset 0, then its mbarrier
+constexpr int kDecodeBarOffset = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
 
 // The image is built with atomic ORs, so it must start as zeros.  Only its front (10 KB, more than most
 // groups need) is cleared up front; a group whose payload turns out longer clears the rest once its size is
@@ -1093,41 +1096,36 @@ __device__ __forceinline__ void prefetch_payload(const StreamView& sv, uint32_t 
     asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
 }
 
-// Stage group payload words [a, a+gw) of the stream into the image.  All of a thread's loads are issued
-// before the first store (a rolled loop would pay one memory round trip per iteration), and they are 128
-// bits wide: the copy starts at the 16-byte boundary at or below word a, so payload word j lands at
-// sm.img[(a & 3) + j] — decode_group reads the image through that shifted origin.
-constexpr int kStageRounds = (kMaxGroupBytes / 4 + 3 + 4 * kThreads - 1) / (4 * kThreads);  // 9
-template <int kRounds>
-__device__ __forceinline__ void stage_rounds(uint4* img4, const uint4* src4, uint32_t n4) {
-  uint4 t[kRounds];
-#pragma unroll
-  for (int r = 0; r < kRounds; ++r)
-    if ((uint32_t)r * kThreads + threadIdx.x < n4) t[r] = __ldcs(src4 + r * kThreads + threadIdx.x);
-#pragma unroll
-  for (int r = 0; r < kRounds; ++r)
-    if ((uint32_t)r * kThreads + threadIdx.x < n4) img4[r * kThreads + threadIdx.x] = t[r];
-}
-__device__ __forceinline__ void stage_payload(Smem& sm, const StreamView& sv) {
+// Stage group payload words [a, a+gw) of the stream into the image.  The copy starts at the 16-byte boundary
+// at or below word a, so payload word j lands at img[(a & 3) + j] — decode_group reads the image through that
+// shifted origin.  Where every 16-byte piece lies inside the stream (all groups but, at most, a stream's
+// last), one thread hands the whole copy to the bulk-copy engine (`cp.async.bulk`, completion on `bar`): no
+// load, no shared-memory store and no register passes through the lanes.  Returns true in that case: after
+// the CTA's next barrier every thread waits with tma_wait_tile(bar).  Otherwise the words are copied by the
+// lanes and the CTA's next barrier completes the staging.
+__device__ __forceinline__ bool stage_payload(uint32_t* img, const StreamView& sv, uint64_t* bar) {
   const uint32_t shift = sv.a & 3u;
   const uint32_t start = sv.a - shift;                // aligned first word
   const uint32_t n_words = sv.gw + shift;             // words to bring in, from the aligned start
   const uint32_t n4 = (n_words + 3u) >> 2;            // 16-byte pieces
   const uint32_t* src = sv.words + (sv.base >> 2) + start;
-  if (start + 4u * n4 <= sv.pw) {                     // every piece lies inside the stream (uniform)
-    const uint4* src4 = reinterpret_cast<const uint4*>(src);
-    uint4* img4 = reinterpret_cast<uint4*>(sm.img);
-    if (n4 <= 3u * kThreads)
-      stage_rounds<3>(img4, src4, n4);
-    else if (n4 <= 5u * kThreads)
-      stage_rounds<5>(img4, src4, n4);
-    else
-      stage_rounds<kStageRounds>(img4, src4, n4);
-  } else {
-    // the last piece would reach past the end of the stream (its last group only): word by word
-#pragma unroll 4
-    for (uint32_t w = threadIdx.x; w < n_words; w += kThreads) sm.img[w] = __ldcs(src + w);
+  if (n4 != 0u && start + 4u * n4 <= sv.pw && (reinterpret_cast<uintptr_t>(src) & 15u) == 0u) {  // uniform
+    if (threadIdx.x == 0) {
+      const uint32_t b = smem_u32(bar), bytes = 16u * n4;
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_proxy_async();
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                       smem_u32(img)),
+                   "l"(src), "r"(bytes), "r"(b)
+                   : "memory");
+    }
+    return true;
   }
+#pragma unroll 4
+  for (uint32_t w = threadIdx.x; w < n_words; w += kThreads) img[w] = __ldcs(src + w);
+  return false;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1212,11 +1210,11 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     nxt_e = __ldg(sv.words + 8 + g + b.prefetch_distance + 1);
   }
   if (ok) {
-    stage_payload(sm, sv);
+    const bool bulk = stage_payload(sm.img, sv, &sm.bar_in);
     prefetch_payload(sv, nxt_a, nxt_e);
-    __syncthreads();  // the image is complete (and the barrier the tile lands on is initialised)
+    __syncthreads();  // lane-copied words are in place; both mbarriers are initialised
     TL(1);
-    if (tma && !tma_wait_tile(&sm.bar)) {
+    if ((bulk && !tma_wait_tile(&sm.bar_in)) || (tma && !tma_wait_tile(&sm.bar))) {
       give_up(b, jg, g, y, kErrTimeout);
       return;
     }
@@ -1276,8 +1274,13 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
   if (ok) {
     // (asking L2 for the payload of the group that will take over this SM slot pays in the fused kernel's
     // mix of loads, not here: 55.6 -> 54.2 us without it)
-    stage_payload(sm, sv);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(dyn_smem + kDecodeBarOffset);  // behind the image and the rows
+    const bool bulk = stage_payload(sm.img, sv, bar);
     __syncthreads();
+    if (bulk && !tma_wait_tile(bar)) {
+      if (threadIdx.x == 0) raise(b.status, kErrTimeout);
+      return;
+    }
     TL(2);
     float mx_unused, mn_unused;
     ok = decode_group<false>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), v, Row{nullptr, 0u}, 0,
@@ -1316,7 +1319,7 @@ __global__ void __launch_bounds__(kThreads, 9) ccoll_decode_kernel(const __grid_
 namespace {
 constexpr int kSmemBytes = kCtlBytes + kRowsBytes;            // fused round: control block + swizzled rows
 constexpr int kSmemCompress = kCtlBytes + kPaddedRowsBytes;  // encoder: control block + padded rows
-constexpr int kSmemDecode = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
+constexpr int kSmemDecode = kDecodeBarOffset + 16;
 
 // Per device: opt in to the dynamic shared-memory size once, and learn how many CTAs of the encoding kernels
 // are resident at a time (the distance of their L2 prefetch).
