@@ -2,19 +2,21 @@
 // include/ccoll.h for the stream layout and the block rules).  Compiled with --fmad=false: every fp32
 // operation of the block rules rounds once, exactly as stated.
 //
-// Lane mapping (all kernels): thread tid of the CTA owns SLICE tid of the group = 32 consecutive values
+// Lane mapping (all kernels): thread tid of the CTA owns ROW tid of the group = 32 consecutive values
 // (128 bytes); block = tid / 4, so four neighbouring lanes share a block and everything that must cross
 // lanes (min/max, the predecessor code, byte offsets) is a two-step shuffle inside that quad of lanes.
 // Per-value work runs serially inside a lane over eight 128-bit quads, so per-block quantities (mid-range,
 // required bits, header) cost 4 lanes, not 32.
 //
-// Data movement: fp32 values enter and leave through shared-memory rows: warps move 512 contiguous bytes per
-// 128-bit load / store instruction and (un)scatter them into per-lane slices padded to 144 bytes, which
-// keeps both the transposing accesses and the lanes' own 128-bit accesses conflict free.  (One 128-byte
+// Data movement: a group's fp32 values are a tile of 128 rows x 128 bytes in shared memory.  In the decoder
+// and the fused round a complete group moves as one TMA tile (cp.async.bulk.tensor, 128-byte swizzle; loads
+// complete on an mbarrier, stores are drained with wait_group.read), and the incoming payload as one bulk
+// copy, so none of it passes through the load/store pipe; the encoder scatters coalesced 128-bit loads into
+// rows padded to 144 bytes instead (cheaper for it than the swizzle's XOR per access).  (One 128-byte
 // bulk-async copy per lane was measured first: a million such copies per 134 MB capped the kernel near
-// 1.2 TB/s, so plain coalesced loads replaced them.)  Variable-length bytes are first appended to the
-// lane's own slice (aligned word stores), then copied once to their byte offset in a shared-memory image
-// of the group's payload, which leaves as coalesced word stores at the offset a decoupled look-back yields.
+// 1.2 TB/s.)  Variable-length bytes are first appended to the lane's own row (aligned word stores), then
+// copied once to their byte offset in a shared-memory image of the group's payload, which leaves as
+// coalesced word stores at the offset that the two-level sum of the earlier groups' sizes yields.
 #include "ccoll_kernels.cuh"
 
 #include <cstring>

@@ -2,7 +2,7 @@
 // compaction (compress), the parallel decoder, and the fused decompress-add-recompress ring round.
 //
 // Work decomposition (all three kernels): one CTA of 128 threads owns one GROUP of 32 blocks (4096 values).
-// Thread t owns slice t = 32 consecutive values, so the four lanes 4b .. 4b+3 share block b.  Per-value
+// Thread t owns row t = 32 consecutive values, so the four lanes 4b .. 4b+3 share block b.  Per-value
 // work runs serially inside a lane; what must cross lanes (min/max, the predecessor code, byte offsets)
 // is a two-step shuffle inside the quad.  Variable-length bytes are staged per lane, copied once into a
 // shared-memory image of the group's payload, and leave the SM as coalesced word stores at the offset
