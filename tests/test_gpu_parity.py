@@ -330,3 +330,58 @@ def test_p2p_allreduce_matches_oracle(P, n):
     ref, ref_moved = ccz.allreduce_sim_p2p(xs, eb)
     got, moved = B.allreduce_sim_p2p(dev(xs), eb)
     assert got.cpu().numpy().tobytes() == ref.tobytes() and moved == ref_moved
+
+
+def test_offset_and_strided_buffers():
+    """Buffers that start 16 bytes into an allocation, rank strides larger than the data and the aliasing
+    stride 0: the tile paths (tensor maps over the caller's buffers) and their plain fallbacks agree."""
+    c = fields.config2(shape=(8, 64, 64), sigma=3.0)              # 32768 values: 8 complete groups
+    x, eb = c["x"].numpy(), float(np.float32(c["eb"]))
+    n = x.size
+    ref_stream = ccz.compress(x, eb)
+    ref_dec = ccz.decompress(ref_stream, n)
+    # input and output 16 bytes into their allocations
+    big_in = torch.zeros(n + 8, device="cuda")
+    big_in[4:4 + n] = dev(x)
+    s = B.compress(big_in[4:4 + n], eb)
+    assert np.array_equal(s.cpu().numpy(), ref_stream)
+    big_out = torch.zeros(n + 8, device="cuda")
+    B.ensure_workspace(n)
+    B.ccoll_decompress(s, s.numel(), n, big_out[4:4 + n])
+    assert B.ccoll_get_status() == B.OK
+    assert big_out[4:4 + n].cpu().numpy().tobytes() == ref_dec.tobytes()
+    assert float(big_out[:4].abs().sum()) == 0.0 and float(big_out[4 + n:].abs().sum()) == 0.0
+    # fused round with the local chunk and the result at such offsets
+    y = np.roll(x, 1000)
+    ref_s2, ref_sum = ccz.reduce_step(ref_stream, y, eb, want_sum=True)
+    big_loc = torch.zeros(n + 8, device="cuda")
+    big_loc[4:4 + n] = dev(y)
+    big_sum = torch.zeros(n + 8, device="cuda")
+    out = torch.empty(B.ccoll_compress_bound(n), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    B.ccoll_reduce_step(s, s.numel(), big_loc[4:4 + n], eb, out, nb, big_sum[4:4 + n])
+    assert B.ccoll_get_status() == B.OK
+    assert np.array_equal(out[: int(nb.item())].cpu().numpy(), ref_s2)
+    assert big_sum[4:4 + n].cpu().numpy().tobytes() == ref_sum.tobytes()
+    assert float(big_sum[:4].abs().sum()) == 0.0 and float(big_sum[4 + n:].abs().sum()) == 0.0
+    # broadcast with a rank stride larger than the data, and with all ranks aliased onto one buffer
+    P = 4
+    ref_bc, _ = ccz.bcast_sim(x, P, eb, mode=0)
+    stride = n + 64
+    B.ensure_workspace(n, P)
+    wide = torch.full((P, stride), -7.0, device="cuda")
+    B.ccoll_bcast_sim(dev(x), wide, stride, P, eb, B.BCAST)
+    assert B.ccoll_get_status() == B.OK
+    assert wide[:, :n].cpu().numpy().tobytes() == ref_bc.tobytes()
+    assert bool((wide[:, n:] == -7.0).all())
+    one = torch.zeros(n, device="cuda")
+    B.ccoll_bcast_sim(dev(x), one, 0, P, eb, B.BCAST)       # contents unspecified by contract, but it must run clean
+    assert B.ccoll_get_status() == B.OK
+    # scatter with a stride larger than the chunk
+    C = B.ccoll_chunk_len(n, P)
+    ref_sc, _ = ccz.bcast_sim(x, P, eb, mode=1)
+    wide = torch.full((P, C + 128), -7.0, device="cuda")
+    B.ccoll_bcast_sim(dev(x), wide, C + 128, P, eb, B.SCATTER)
+    assert B.ccoll_get_status() == B.OK
+    assert wide[:, :C].cpu().numpy().tobytes() == ref_sc.tobytes()
+    assert bool((wide[:, C:] == -7.0).all())
