@@ -66,6 +66,22 @@ __device__ __forceinline__ float min3_nan(float a, float b, float c) {
   asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+// Byte permutation with a selector that is known to be well formed (every nibble 0..7): the intrinsic
+// __byte_perm masks a run-time selector first, one more integer instruction per use.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+__device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t opaque(uint32_t v) {  // hides a constant from the optimiser
+  asm("" : "+r"(v));
+  return v;
+}
 __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t* p) {
   uint64_t v;
   asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -263,6 +279,7 @@ __device__ __forceinline__ void tma_load_tile(const CUtensorMap* map, uint8_t* r
 // false = it gave up (the caller raises a time-out and does not touch the rows).
 __device__ __forceinline__ bool tma_wait_tile(uint64_t* bar) {
   const uint32_t b = smem_u32(bar);
+#pragma unroll 1
   for (uint32_t tries = 0; tries < (1u << 16); ++tries) {
     uint32_t done;
     asm volatile(
@@ -1054,12 +1071,13 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
     const uint32_t msh = 1u << sh;  // q << sh == q * 2^sh
     const uint32_t kSel01 = 0x32143210u, kSel23 = 0x34563245u;  // byte selectors for nb = 0, 1 | 2, 3
     const uint32_t kPick = 0x10u + 0x22u * B;                   // picks table entry nb = B - lead
+    const uint32_t m8 = opaque(0u - 8u);  // a multiplier the compiler cannot see: c = c8B - 8 l stays ONE multiply-add
 #pragma unroll kUnroll
     for (int j = 0; j < 8; ++j) {
       const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
       const uint32_t l0 = cb & 3u, l1 = (cb >> 2) & 3u, l2 = (cb >> 4) & 3u, l3 = cb >> 6;
-      const uint32_t c0 = c8B - 8u * l0, c1 = c8B - 8u * l1, c2 = c8B - 8u * l2;
-      const uint32_t wi = pos >> 2, z = 8u * (pos & 3u);
+      const uint32_t c0 = mad_lo(l0, m8, c8B), c1 = mad_lo(l1, m8, c8B), c2 = mad_lo(l2, m8, c8B);  // 8 * stored bytes
+      const uint32_t wi = pos >> 2, z = 8u * pos;  // the funnel shifts use z mod 32 = 8 * (pos & 3)
       const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3];
       // at most 12 bytes per quad here: three words of string are enough
       const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z);
@@ -1068,10 +1086,10 @@ __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, con
       const uint32_t X0 = __funnelshift_r(U0, U1, c1);
       const uint32_t X1 = __funnelshift_r(U1, S2 >> c0, c1);
       const uint32_t r3 = __funnelshift_r(X0, X1, c2);
-      const uint32_t q0 = __byte_perm(prev, S0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l0));
-      const uint32_t q1 = __byte_perm(q0, U0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l1));
-      const uint32_t q2 = __byte_perm(q1, X0, __byte_perm(kSel01, kSel23, kPick - 0x22u * l2));
-      const uint32_t q3 = __byte_perm(q2, r3, __byte_perm(kSel01, kSel23, kPick - 0x22u * l3));
+      const uint32_t q0 = prmt(prev, S0, prmt(kSel01, kSel23, kPick - 0x22u * l0));
+      const uint32_t q1 = prmt(q0, U0, prmt(kSel01, kSel23, kPick - 0x22u * l1));
+      const uint32_t q2 = prmt(q1, X0, prmt(kSel01, kSel23, kPick - 0x22u * l2));
+      const uint32_t q3 = prmt(q2, r3, prmt(kSel01, kSel23, kPick - 0x22u * l3));
       prev = q3;
       put(j, make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
                          __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu)));
