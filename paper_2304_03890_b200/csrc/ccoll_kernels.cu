@@ -19,6 +19,7 @@
 // coalesced word stores at the offset that the two-level sum of the earlier groups' sizes yields.
 #include "ccoll_kernels.cuh"
 
+#include <cstdlib>
 #include <cstring>
 
 #include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; nothing links libcuda)
@@ -1346,7 +1347,7 @@ constexpr int kSmemDecode = kDecodeBarOffset + 16;
 // Per device: opt in to the dynamic shared-memory size once, and learn how many CTAs of the encoding kernels
 // are resident at a time (the distance of their L2 prefetch).
 bool g_ready[64];
-uint32_t g_slots[64], g_slots_decode[64];
+uint32_t g_slots[64];
 // Tensor map of a buffer seen as [32 fp32][rows][planes] with 128-byte rows, tile = 32 x 128 x 1, 128-byte
 // swizzle.  The encoder is a driver entry point looked up once through the runtime.  False if it cannot be
 // had or refuses the arguments: the kernels then use their plain load/store paths.
@@ -1362,7 +1363,8 @@ bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t p
       fn = nullptr;
     return reinterpret_cast<EncodeTiledFn>(fn);
   }();
-  if (!encode || (reinterpret_cast<uintptr_t>(base) & 15u)) return false;
+  static const bool disabled = std::getenv("CCOLL_NO_TMA") != nullptr;  // forces the plain load/store paths (tests)
+  if (disabled || !encode || (reinterpret_cast<uintptr_t>(base) & 15u)) return false;
   if (planes > 1 && ((plane_stride_bytes & 15u) || plane_stride_bytes >= (1ull << 40))) return false;
   const cuuint64_t dims[3] = {32u, rows, planes ? planes : 1u};
   const cuuint64_t strides[2] = {128u, planes > 1 ? plane_stride_bytes : 128u * rows};
@@ -1386,9 +1388,6 @@ bool device_ready() {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_compress_kernel, kThreads, kSmemCompress) != cudaSuccess)
       return false;
     g_slots[dev] = (uint32_t)(sms * (per_sm > 0 ? per_sm : 1));
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ccoll_decode_kernel, kThreads, kSmemDecode) != cudaSuccess)
-      return false;
-    g_slots_decode[dev] = (uint32_t)(sms * (per_sm > 0 ? per_sm : 1));
     g_ready[dev] = true;
   }
   return true;
@@ -1430,11 +1429,7 @@ bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cuda
 }
 bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
   if (!device_ready()) return false;
-  int dev = 0;
-  cudaGetDevice(&dev);
   DecodeBatch b = b0;
-  const uint32_t streams = jobs * ranks;  // CTAs are issued x-fastest over (group, stream, rank)
-  b.prefetch_distance = streams == 1 ? g_slots_decode[dev] : (g_slots_decode[dev] + streams - 1) / streams;
   // The output as a tensor of 128-byte rows: [32 values][rows of a destination][destinations].
   CUtensorMap map;
   std::memset(&map, 0, sizeof(map));

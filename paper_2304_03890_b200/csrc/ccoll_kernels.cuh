@@ -81,7 +81,6 @@ struct DecodeBatch {
                    // 4: one destination per chunk, rank (y + rot) mod P (grid.z = 1)
   int rot;
   int scatter;     // 1: job y writes at out + y*out_rank_stride; 0: at out + z*out_rank_stride + y*C
-  uint32_t prefetch_distance;  // groups ahead whose payload a CTA asks L2 for (set by the launcher)
   int use_tma;                 // complete groups leave through the TMA unit (set by the launcher)
   uint32_t* status;
 };

@@ -385,3 +385,31 @@ def test_offset_and_strided_buffers():
     assert B.ccoll_get_status() == B.OK
     assert wide[:, :C].cpu().numpy().tobytes() == ref_sc.tobytes()
     assert bool((wide[:, C:] == -7.0).all())
+
+
+def test_plain_paths_without_the_tma_unit(tmp_path):
+    """CCOLL_NO_TMA=1 makes the library skip its tensor maps, so complete groups also take the plain
+    load/store paths that ragged groups (and a driver without the encoder entry point) use."""
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_2304_03890_b200 import binding as B, fields\n"
+        "from oracle import ccz\n"
+        "c = fields.config3(P=4, shape=(32, 32, 40), sigma=3.0)\n"
+        "xs, eb = c['x'].numpy(), float(np.float32(c['eb']))\n"
+        "x = xs[0]\n"
+        "s = B.compress(torch.from_numpy(x).cuda(), eb)\n"
+        "assert np.array_equal(s.cpu().numpy(), ccz.compress(x, eb))\n"
+        "d = B.decompress(s, x.size)\n"
+        "assert d.cpu().numpy().tobytes() == ccz.decompress(ccz.compress(x, eb), x.size).tobytes()\n"
+        "ref, moved = ccz.allreduce_sim(xs, eb)\n"
+        "got, gm = B.allreduce_sim(torch.from_numpy(xs).cuda(), eb)\n"
+        "assert got.cpu().numpy().tobytes() == ref.tobytes() and gm == moved\n"
+        "print('plain ok')\n"
+    )
+    import os
+    env = dict(os.environ, CCOLL_NO_TMA="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "plain ok" in r.stdout, r.stdout + r.stderr
