@@ -218,6 +218,8 @@ __device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg
 // are only 128 bytes apart (no padding).  Byte offset o < 128 of row t is at  128 t + (o ^ 16 (t & 7))  =
 // (128 t + 16 (t & 7)) ^ o : one XOR per access.
 struct Row {
+  static constexpr uint32_t kWords = 32u;  // words a lane may stage into
+  __device__ static __forceinline__ uint32_t rot(uint32_t) { return 0u; }
   uint8_t* tile;  // the rows buffer (1024-byte aligned)
   uint32_t off;   // 128 t + 16 (t & 7)
   __device__ __forceinline__ float4 quad(uint32_t j) const {
@@ -244,6 +246,10 @@ __device__ __forceinline__ Row row_of(uint8_t* rows, uint32_t t) { return Row{ro
 constexpr int kPaddedRowBytes = 144;
 constexpr int kPaddedRowsBytes = kThreads * kPaddedRowBytes;  // 18432
 struct PaddedRow {
+  static constexpr uint32_t kWords = 36u;
+  // Staged words start `rot` words into the row: with rows 36 words apart, lanes l and l + 8 would otherwise
+  // hit the same bank whenever they are at the same word; lane l's word w now sits in bank 4 l + l/8 + w.
+  __device__ static __forceinline__ uint32_t rot(uint32_t t) { return (t >> 3) & 3u; }
   uint8_t* p;
   __device__ __forceinline__ float4 quad(uint32_t j) const { return *reinterpret_cast<const float4*>(p + 16u * j); }
   __device__ __forceinline__ uint4 words4(uint32_t j) const { return *reinterpret_cast<const uint4*>(p + 16u * j); }
@@ -471,6 +477,7 @@ __device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t 
   const float mu = __uint_as_float(mu_bits);
   uint32_t lo = 0u, hi = 0u, Tb = 0u;
   uint32_t clo = 0u, chi = 0u;
+  const uint32_t rot = RowT::rot(threadIdx.x);  // staged word k goes to word rot + k of the row
   auto put = [&](uint32_t q, uint32_t sa) {
     const uint32_t n = 32u - sa;
     const uint32_t t = __funnelshift_lc(0u, q, sa);  // the stored bits, at the top of the word
@@ -478,12 +485,16 @@ __device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t 
     hi = __funnelshift_lc(lo, hi, n);
     lo = __funnelshift_lc(t, lo, n);
     if ((Tn ^ Tb) & 32u)  // a word boundary was crossed (n <= 32: at most one)
-      row.set_word((Tn >> 5) - 1u, __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123));
+      row.set_word(rot + (Tn >> 5) - 1u, __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123));
     Tb = Tn;
   };
+  // the next quad is always read before the current one's words are stored: they may reach rot <= 3 words
+  // into it
+  float4 xn = row.quad(0);
 #pragma unroll(kGeneral ? 1 : 2)
   for (int j = 0; j < 8; ++j) {
-    const float4 x = row.quad(j);
+    const float4 x = xn;
+    xn = row.quad(j < 7 ? j + 1 : 7);
     const uint32_t q0 = __float_as_uint(lossless ? x.x : __fsub_rn(x.x, mu)) >> sh,
                    q1 = __float_as_uint(lossless ? x.y : __fsub_rn(x.y, mu)) >> sh,
                    q2 = __float_as_uint(lossless ? x.z : __fsub_rn(x.z, mu)) >> sh,
@@ -514,8 +525,8 @@ __device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t 
   const uint32_t pend = Tb & 31u, w = Tb >> 5;
   // the last partial word, zero padded, and a zero word behind it for the realigning copy — as far as the row
   // reaches (a row that is full to its last byte has neither; copy_staged reads zeros past the row's end)
-  if (w < 32u) row.set_word(w, pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u);
-  if (w + 1u < 32u) row.set_word(w + 1u, 0u);
+  if (rot + w < RowT::kWords) row.set_word(rot + w, pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u);
+  if (rot + w + 1u < RowT::kWords) row.set_word(rot + w + 1u, 0u);
   T_out = Tb >> 3;
   code_lo = clo;
   code_hi = chi;
@@ -526,32 +537,37 @@ __device__ __noinline__ void emit_lane_general(RowT row, uint32_t R, uint32_t mu
   emit_lane<true, RowT>(row, R, mu_bits, nv, prev, T_out, code_lo, code_hi);
 }
 
-// Copy the lane's T staged bytes from its row to byte offset dst of the image.  The first and last image
-// word may be shared with a neighbour and are ORed in; the words between are plain stores.
+// Copy the lane's T staged bytes (they start at word rot of its row) to byte offset dst of the image.  The
+// first and last image word may be shared with a neighbour and are ORed in; the words between are plain
+// stores.  The row is read in aligned 128-bit pieces from its start, as a string whose first rot words are
+// to be skipped: row word g goes to image word (dst / 4) - rot + g.
 template <class RowT>
 __device__ __forceinline__ void copy_staged(uint32_t* img, const RowT& row, uint32_t dst, uint32_t T) {
   if (T == 0u) return;
+  const uint32_t rot = RowT::rot(threadIdx.x);
   const uint32_t z = 8u * (dst & 3u);
-  uint32_t* out = img + (dst >> 2);
+  uint32_t* out = img + (dst >> 2);                // image word of staged word 0
   const uint32_t nw = ((dst & 3u) + T + 3u) >> 2;  // image words touched, <= 33
-  atomicOr(&out[0], row.word(0) << z);
+  atomicOr(&out[0], row.word(rot) << z);
   if (nw > 1u) {
-    const uint32_t last = nw - 1u < 32u ? row.word(nw - 1u) : 0u;  // nothing is staged past the row's 32 words
-    atomicOr(&out[nw - 1u], __funnelshift_l(row.word(nw - 2u), last, z));
+    const uint32_t k = rot + nw - 1u;  // nothing is staged past the row's last word
+    const uint32_t last = k < RowT::kWords ? row.word(k) : 0u;
+    atomicOr(&out[nw - 1u], __funnelshift_l(row.word(k - 1u), last, z));
   }
   if (nw <= 2u) return;
-  const uint32_t ni = nw - 2u;  // interior words 1 .. nw-2
+  const uint32_t ni = nw - 2u;  // interior image words 1 .. nw-2 = row words rot+1 .. rot+nw-2
+  uint32_t* outr = out - rot;   // image word of row word 0 (never dereferenced below row word rot + 1)
   uint32_t prevw = 0u;
-  for (uint32_t c = 0; 4u * c <= ni; ++c) {
+  for (uint32_t c = 0; 4u * c <= rot + ni; ++c) {
     const uint4 cur = row.words4(c);
     const uint32_t w0 = __funnelshift_l(prevw, cur.x, z), w1 = __funnelshift_l(cur.x, cur.y, z),
                    w2 = __funnelshift_l(cur.y, cur.z, z), w3 = __funnelshift_l(cur.z, cur.w, z);
     prevw = cur.w;
-    const uint32_t g = 4u * c;  // image word of w0; word g is interior iff g - 1 < ni (unsigned)
-    if (g - 1u < ni) out[g] = w0;
-    if (g < ni) out[g + 1u] = w1;
-    if (g + 1u < ni) out[g + 2u] = w2;
-    if (g + 2u < ni) out[g + 3u] = w3;
+    const uint32_t g = 4u * c - rot;  // staged word index of cur.x (wraps below zero for skipped words)
+    if (g - 1u < ni) outr[4u * c] = w0;
+    if (g < ni) outr[4u * c + 1u] = w1;
+    if (g + 1u < ni) outr[4u * c + 2u] = w2;
+    if (g + 2u < ni) outr[4u * c + 3u] = w3;
   }
 }
 
