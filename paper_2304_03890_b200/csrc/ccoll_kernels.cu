@@ -218,8 +218,6 @@ __device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg
 // are only 128 bytes apart (no padding).  Byte offset o < 128 of row t is at  128 t + (o ^ 16 (t & 7))  =
 // (128 t + 16 (t & 7)) ^ o : one XOR per access.
 struct Row {
-  static constexpr uint32_t kWords = 32u;  // words a lane may stage into
-  __device__ static __forceinline__ uint32_t rot(uint32_t) { return 0u; }
   uint8_t* tile;  // the rows buffer (1024-byte aligned)
   uint32_t off;   // 128 t + 16 (t & 7)
   __device__ __forceinline__ float4 quad(uint32_t j) const {
@@ -228,21 +226,14 @@ struct Row {
   __device__ __forceinline__ void set_quad(uint32_t j, const float4& v) const {
     *reinterpret_cast<float4*>(tile + (off ^ (16u * j))) = v;
   }
-  __device__ __forceinline__ uint4 words4(uint32_t j) const {
-    return *reinterpret_cast<const uint4*>(tile + (off ^ (16u * j)));
-  }
-  __device__ __forceinline__ uint32_t word(uint32_t i) const {
-    return *reinterpret_cast<const uint32_t*>(tile + (off ^ (4u * i)));
-  }
-  __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const {
-    *reinterpret_cast<uint32_t*>(tile + (off ^ (4u * i))) = v;
-  }
 };
 __device__ __forceinline__ Row row_of(uint8_t* rows, uint32_t t) { return Row{rows, 128u * t + 16u * (t & 7u)}; }
 // The other way to keep a lane's walk over its row free of bank conflicts: rows 144 bytes apart, no swizzle, no
-// XOR.  The TMA unit cannot produce it (a tile is dense), so the values are (un)scattered by the lanes.  The
-// encoder alone, whose integer pipe is its busiest unit, is faster this way; where a tile also has to leave
-// again (decoder, fused round) the swizzled rows win.  Same interface as Row.
+// XOR per access.  The TMA unit makes this layout too: a box 36 values wide over a tensor whose rows have 32
+// lands as rows of 144 bytes (the four values past the row's end are out of bounds and arrive as zeros; a
+// store does not write them).  The encoder and the fused round use it (their integer pipe is the busy one,
+// and the spare words of a row let lanes stagger their staged output); the decoder's output tile is swizzled
+// (16 KB instead of 18 KB: that is what lets 12 of its CTAs share an SM).  Same interface as Row.
 constexpr int kPaddedRowBytes = 144;
 constexpr int kPaddedRowsBytes = kThreads * kPaddedRowBytes;  // 18432
 struct PaddedRow {
@@ -252,14 +243,13 @@ struct PaddedRow {
   __device__ static __forceinline__ uint32_t rot(uint32_t t) { return (t >> 3) & 3u; }
   uint8_t* p;
   __device__ __forceinline__ float4 quad(uint32_t j) const { return *reinterpret_cast<const float4*>(p + 16u * j); }
+  __device__ __forceinline__ void set_quad(uint32_t j, const float4& v) const { *reinterpret_cast<float4*>(p + 16u * j) = v; }
   __device__ __forceinline__ uint4 words4(uint32_t j) const { return *reinterpret_cast<const uint4*>(p + 16u * j); }
   __device__ __forceinline__ uint32_t word(uint32_t i) const { return *reinterpret_cast<const uint32_t*>(p + 4u * i); }
   __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const { *reinterpret_cast<uint32_t*>(p + 4u * i) = v; }
 };
 template <class RowT>
 __device__ __forceinline__ RowT make_row(uint8_t* rows, uint32_t t);
-template <>
-__device__ __forceinline__ Row make_row<Row>(uint8_t* rows, uint32_t t) { return row_of(rows, t); }
 template <>
 __device__ __forceinline__ PaddedRow make_row<PaddedRow>(uint8_t* rows, uint32_t t) {
   return PaddedRow{rows + kPaddedRowBytes * t};
@@ -270,12 +260,12 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // One thread: arm the barrier and ask the TMA unit for rows [row0, row0+128) of plane `plane` of the tensor.
 __device__ __forceinline__ void tma_load_tile(const CUtensorMap* map, uint8_t* rows, uint64_t* bar, uint32_t row0,
-                                              uint32_t plane) {
+                                              uint32_t plane, uint32_t tile_bytes) {
   const uint32_t b = smem_u32(bar);
   asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   fence_proxy_async();
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(kRowsBytes) : "memory");
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(tile_bytes) : "memory");
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
           smem_u32(rows)),
@@ -339,30 +329,9 @@ __device__ __forceinline__ void load_rows_padded(uint8_t* rows, const float* x, 
     dst[r * kRoundStride] = v;
   }
 }
-// The same tile without the TMA unit (a group that is not complete, or no tensor map): coalesced 128-bit
-// loads, bounds watched, zeros past the end; thread tid moves the float4 number r*128 + tid in round r, which
-// is piece (tid & 7) of row 16 r + tid / 8.  A __syncthreads must follow before the rows are read.
-__device__ __forceinline__ void load_rows(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
-  const uint32_t tid = threadIdx.x;
-  const uint32_t cnt = group_count(jg, g);
-  const float* src = x + (size_t)g * kGroupValues;
-  uint8_t* dst = rows + 128u * (tid >> 3) + 16u * ((tid & 7u) ^ ((tid >> 3) & 7u));
-#pragma unroll 1
-  for (int r = 0; r < 8; ++r) {
-    const uint32_t f = (uint32_t)r * kThreads + tid;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (4u * f + 4u <= cnt) {
-      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
-    } else {
-      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
-      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
-      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
-    }
-    *reinterpret_cast<float4*>(dst + 2048 * r) = v;
-  }
-}
-// ... and out: coalesced 128-bit streaming stores from the rows, bounds watched.  A __syncthreads must
-// separate it from the writes of the rows.
+// A swizzled tile without the TMA unit (a group that is not complete, or no tensor map): coalesced 128-bit
+// streaming stores, bounds watched; thread tid moves the float4 number r*128 + tid in round r, which is piece
+// (tid & 7) of row 16 r + tid / 8.  A __syncthreads must separate it from the writes of the rows.
 __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
   const uint32_t tid = threadIdx.x;
   const uint32_t cnt = group_count(jg, g);
@@ -372,6 +341,26 @@ __device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, cons
   for (int r = 0; r < 8; ++r) {
     const uint32_t f = (uint32_t)r * kThreads + tid;
     const float4 t = *reinterpret_cast<const float4*>(src + 2048 * r);
+    if (4u * f + 4u <= cnt) {
+      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+    } else {
+      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
+      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
+      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+    }
+  }
+}
+// The same from padded rows (fused round: the owner's sums of a group that is not complete).
+__device__ __forceinline__ void store_rows_padded(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint32_t cnt = group_count(jg, g);
+  float* dst = out + (size_t)g * kGroupValues;
+  const float4* src = reinterpret_cast<const float4*>(rows + (tid >> 3) * kPaddedRowBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kPaddedRowBytes / 16;
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    const float4 t = src[r * kRoundStride];
     if (4u * f + 4u <= cnt) {
       __stcs(reinterpret_cast<float4*>(dst) + f, t);
     } else {
@@ -942,9 +931,9 @@ __device__ __forceinline__ float reduce_op(float a, float b, int op, float divis
 // each decoded quad is REDUCED (op) with the quad of local values waiting in the lane's slice and the result is written
 // back there, and mx / mn receive the largest / smallest result of the lane (meaningless for a ragged slice);
 // the loops are then unrolled only twice, which keeps the fused kernel inside the instruction cache.
-template <bool kToSlice, bool kDivide = false>
+template <bool kToSlice, bool kDivide = false, class RowT = Row>
 __device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
-                                             float4 (&v)[8], const Row& row, int op, float divisor, float& mx,
+                                             float4 (&v)[8], const RowT& row, int op, float divisor, float& mx,
                                              float& mn) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
@@ -1193,6 +1182,9 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __gri
   const float* x = b.x + (uint64_t)rank * b.x_rank_stride + jg.lo;
   const LaneGeom lg = lane_geom(jg, g);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
+  // (A TMA tile load into these rows was measured too: 78 us against 71 us.  Nothing else can run in this CTA
+  // until its values are there, and the one bulk request comes back later than eight rounds of plain loads; in
+  // the fused round the same tile load hides behind the staging of the payload and wins.)
   load_rows_padded(rows, x, jg, g);
   prefetch_group(x, jg, g + b.prefetch_distance);
   zero_image(sm.img);
@@ -1223,14 +1215,14 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const LaneGeom lg = lane_geom(jg, g);
   TL(0);
   const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
-  const Row row = row_of(rows, threadIdx.x);
-  const bool whole = group_count(jg, g) == (uint32_t)kGroupValues && (smem_u32(rows) & 1023u) == 0u;
+  const PaddedRow row = make_row<PaddedRow>(rows, threadIdx.x);
+  const bool whole = group_count(jg, g) == (uint32_t)kGroupValues;
   const bool tma = b.use_tma_in && whole;
   const uint32_t row0 = (jg.lo + g * (uint32_t)kGroupValues) >> 5;  // the group's first row in the rank buffer
   if (tma) {
-    if (threadIdx.x == 0) tma_load_tile(&x_map, rows, &sm.bar, row0, b.x_rank_stride ? rank : 0u);
+    if (threadIdx.x == 0) tma_load_tile(&x_map, rows, &sm.bar, row0, b.x_rank_stride ? rank : 0u, kPaddedRowsBytes);
   } else {
-    load_rows(rows, local, jg, g);
+    load_rows_padded(rows, local, jg, g);
   }
   prefetch_group(local, jg, g + b.prefetch_distance);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
@@ -1256,7 +1248,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
       return;
     }
     // decoded (op) local, one rounded operation per value, left in the lane's row
-    ok = decode_group<true, kDivide>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, row,
+    ok = decode_group<true, kDivide, PaddedRow>(sm, sv, lg, min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks), unused, row,
                                      b.op, b.divisor, mx, mn);
   }
   TL(2);
@@ -1273,16 +1265,16 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
     if (tma_sum) {
       if (threadIdx.x == 0) tma_store_tile(&sum_map, rows, row0, b.sum_rank_stride ? rank : 0u);
     } else {
-      store_rows(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
+      store_rows_padded(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
     }
     __syncthreads();  // the rows are about to be reused for staging
   }
   TL(3);
   if (tail) {
-    pad_ragged<Row>(rows, lg);
+    pad_ragged<PaddedRow>(rows, lg);
     lane_minmax(row, mx, mn);
   }
-  encode_group<Row>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
+  encode_group<PaddedRow>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
   TL(7);
 }
 
@@ -1356,8 +1348,8 @@ __global__ void __launch_bounds__(kThreads, 12) ccoll_decode_kernel(const __grid
 }  // namespace
 
 namespace {
-constexpr int kSmemBytes = kCtlBytes + kRowsBytes;            // fused round: control block + swizzled rows
-constexpr int kSmemCompress = kCtlBytes + kPaddedRowsBytes;  // encoder: control block + padded rows
+constexpr int kSmemBytes = kCtlBytes + kPaddedRowsBytes;  // encoder and fused round: control block + padded rows
+constexpr int kSmemCompress = kSmemBytes;
 constexpr int kSmemDecode = kDecodeBarOffset + 16;
 
 // Per device: opt in to the dynamic shared-memory size once, and learn how many CTAs of the encoding kernels
@@ -1370,7 +1362,8 @@ uint32_t g_slots[64];
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes) {
+bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes,
+                   bool padded) {
   static EncodeTiledFn encode = [] {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
@@ -1384,11 +1377,13 @@ bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t p
   if (planes > 1 && ((plane_stride_bytes & 15u) || plane_stride_bytes >= (1ull << 40))) return false;
   const cuuint64_t dims[3] = {32u, rows, planes ? planes : 1u};
   const cuuint64_t strides[2] = {128u, planes > 1 ? plane_stride_bytes : 128u * rows};
-  const cuuint32_t box[3] = {32u, 128u, 1u};
+  // padded: a box 36 values wide over rows of 32 -> shared-memory rows of 144 bytes, the last four values out of
+  // bounds (zeros on a load, not written by a store); otherwise dense rows with the 128-byte swizzle
+  const cuuint32_t box[3] = {padded ? (cuuint32_t)(kPaddedRowBytes / 4) : 32u, 128u, 1u};
   const cuuint32_t estr[3] = {1u, 1u, 1u};
   return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                CU_TENSOR_MAP_INTERLEAVE_NONE, padded ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool device_ready() {
@@ -1423,7 +1418,8 @@ static EncodeBatch with_prefetch(const EncodeBatch& b, uint32_t jobs) {
 // The fp32 side of an encode batch as a tensor of 128-byte rows: [32 values][rows of a rank][ranks].
 static bool rank_buffer_map(CUtensorMap* map, const float* base, uint64_t n, uint64_t rank_stride, int P) {
   std::memset(map, 0, sizeof(*map));
-  return base && n / 32u >= 128u && make_tile_map(map, base, n / 32u, rank_stride ? (uint64_t)P : 1u, rank_stride * 4u);
+  return base && n / 32u >= 128u &&
+         make_tile_map(map, base, n / 32u, rank_stride ? (uint64_t)P : 1u, rank_stride * 4u, /*padded=*/true);
 }
 bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
   if (!device_ready()) return false;
@@ -1451,7 +1447,7 @@ bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint
   std::memset(&map, 0, sizeof(map));
   const uint64_t rows = (b.scatter ? b.chunk_len : b.n) / 32u;
   const uint64_t planes = b.out_rank_stride ? (b.scatter ? jobs : (b.skip_mode == 4 ? (uint32_t)b.P : ranks)) : 1u;
-  b.use_tma = rows >= 128u && make_tile_map(&map, b.out, rows, planes, b.out_rank_stride * 4u) ? 1 : 0;
+  b.use_tma = rows >= 128u && make_tile_map(&map, b.out, rows, planes, b.out_rank_stride * 4u, /*padded=*/false) ? 1 : 0;
   ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b, map);
   return true;
 }
