@@ -413,3 +413,48 @@ def test_plain_paths_without_the_tma_unit(tmp_path):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "plain ok" in r.stdout, r.stdout + r.stderr
+
+
+def test_seeded_fuzz_against_the_oracle():
+    """Many small seeded cases of mixed character (smooth, noisy, constant stretches, spikes, denormals, huge and
+    tiny magnitudes, NaN / Inf) and random sizes and bounds: streams, decoded values and one fused round must
+    equal the oracle's bit for bit."""
+    rng = np.random.default_rng(20230403)
+    for case in range(240):
+        n = int(rng.choice([rng.integers(1, 300), rng.integers(300, 5000), rng.integers(5000, 20000)]))
+        kind = case % 6
+        t = np.arange(n, dtype=np.float64)
+        if kind == 0:
+            x = np.sin(t * rng.uniform(1e-3, 0.3)) * rng.uniform(0.1, 1e3)
+        elif kind == 1:
+            x = rng.standard_normal(n) * 10.0 ** rng.uniform(-8, 8)
+        elif kind == 2:
+            x = np.repeat(rng.standard_normal(n // 97 + 1), 97)[:n] + (rng.random(n) < 0.01) * rng.standard_normal(n)
+        elif kind == 3:
+            x = np.cumsum(rng.standard_normal(n)) * 10.0 ** rng.uniform(-3, 3)
+        elif kind == 4:
+            x = rng.standard_normal(n) * 1e-41                      # denormals
+        else:
+            x = np.where(rng.random(n) < 0.5, 0.0, rng.standard_normal(n) * 1e30)
+        x = x.astype(np.float32)
+        if case % 5 == 0 and n > 3:
+            idx = rng.integers(0, n, size=3)
+            x[idx[0]] = np.nan
+            x[idx[1]] = np.inf
+            x[idx[2]] = -np.inf
+        finite = x[np.isfinite(x)]
+        span = float(finite.max() - finite.min()) if finite.size else 1.0
+        eb = float(np.float32(max(span, 1e-30) * 10.0 ** rng.uniform(-7, -0.5)))
+        if not (eb > 0 and np.isfinite(eb)):
+            eb = 1e-3
+        ref = ccz.compress(x, eb)
+        got = B.compress(dev(x), eb)
+        assert np.array_equal(got.cpu().numpy(), ref), (case, n, eb)
+        dec = B.decompress(got, n).cpu().numpy()
+        assert dec.tobytes() == ccz.decompress(ref, n).tobytes(), (case, n, eb)
+        y = np.roll(x, 7).copy()
+        y[~np.isfinite(y)] = 1.0
+        r_ref, s_ref = ccz.reduce_step(ref, y, eb, want_sum=True)
+        r_got, s_got = B.reduce_step(got, dev(y), eb, want_sum=True)
+        assert np.array_equal(r_got.cpu().numpy(), r_ref), (case, n, eb)
+        assert s_got.cpu().numpy().tobytes() == s_ref.tobytes(), (case, n, eb)
