@@ -336,19 +336,45 @@ def main():
     e2e_steps = max(2, min(args.steps, 10))
     d2h = 0
 
+    # The copies run on streams of their own, ordered against the calls by events: x2 goes up while compress and
+    # decompress run, and every result starts down as soon as its call has finished (PCIe carries both ways).
+    s_in, s_out, cur = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    ev = [torch.cuda.Event() for _ in range(8)]
+
     def e2e_step():
         nonlocal d2h
-        x.copy_(hx, non_blocking=True)
-        x2.copy_(hx2, non_blocking=True)
-        step()
-        h_nb.copy_(nb1, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        sb = int(h_nb.item())
-        h_s1[:sb].copy_(s1[:sb], non_blocking=True)
-        h_dec.copy_(dec, non_blocking=True)
-        h_sum.copy_(ssum, non_blocking=True)
-        h_ar.copy_(ar_out, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        s_in.wait_stream(cur)      # the previous step's calls are done with x and x2
+        s_out.wait_stream(cur)
+        with torch.cuda.stream(s_in):
+            x.copy_(hx, non_blocking=True)
+            ev[0].record(s_in)
+            x2.copy_(hx2, non_blocking=True)
+            ev[1].record(s_in)
+        cur.wait_event(ev[0])
+        B.ccoll_compress(x, eb, s1, nb1)
+        ev[2].record(cur)
+        B.ccoll_decompress(s1, in_bytes, n, dec)
+        ev[3].record(cur)
+        cur.wait_event(ev[1])
+        B.ccoll_reduce_step(s1, in_bytes, x2, eb, s2, nb2, ssum)
+        ev[4].record(cur)
+        B.ccoll_allreduce_sim(xr, ar_out.view(P, n // P), eb, moved)
+        ev[5].record(cur)
+        B.ccoll_bcast_sim(x, sc_out, C, P, eb, B.SCATTER, cb)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev[2])
+            h_nb.copy_(nb1, non_blocking=True)
+            s_out.synchronize()
+            sb = int(h_nb.item())
+            h_s1[:sb].copy_(s1[:sb], non_blocking=True)
+            s_out.wait_event(ev[3])
+            h_dec.copy_(dec, non_blocking=True)
+            s_out.wait_event(ev[4])
+            h_sum.copy_(ssum, non_blocking=True)
+            s_out.wait_event(ev[5])
+            h_ar.copy_(ar_out, non_blocking=True)
+        s_out.synchronize()
+        cur.synchronize()
         d2h = sb + 3 * 4 * n + 8
 
     e2e_step()
