@@ -288,15 +288,15 @@ __device__ __forceinline__ bool tma_wait_tile(uint64_t* bar) {
   }
   return false;
 }
-// One thread: store the tile to rows [row0, row0+128) of plane `plane` of the tensor, and wait until shared
-// memory has been read (the CTA may then exit or reuse it).
+// One thread: store the tile to rows [row0, row0+128) of plane `plane` of the tensor; the same thread then
+// calls tma_store_wait() before shared memory is reused or the CTA exits (the tile has been read by then).
 __device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, const uint8_t* rows, uint32_t row0, uint32_t plane) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
                "r"(row0), "r"(plane), "r"(smem_u32(rows))
                : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
+__device__ __forceinline__ void tma_store_wait() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // Padded rows: every warp reads 512 contiguous bytes per instruction (128-bit streaming loads) and scatters
 // them; in round r thread tid moves the float4 number r*128 + tid of the group, piece (tid & 7) of row
@@ -1260,10 +1260,11 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   const bool tma_sum = b.sum_out && b.use_tma_sum && whole;
   if (tma_sum) fence_proxy_async();  // the results just written are about to be read by the TMA unit
   __syncthreads();  // every thread is done reading the incoming image (and has written its results)
-  zero_image(sm.img);
+  if (tma_sum && threadIdx.x == 0) tma_store_tile(&sum_map, rows, row0, b.sum_rank_stride ? rank : 0u);
+  zero_image(sm.img);  // while the TMA unit reads the tile
   if (b.sum_out) {
     if (tma_sum) {
-      if (threadIdx.x == 0) tma_store_tile(&sum_map, rows, row0, b.sum_rank_stride ? rank : 0u);
+      if (threadIdx.x == 0) tma_store_wait();
     } else {
       store_rows_padded(rows, b.sum_out + (uint64_t)rank * b.sum_rank_stride + jg.lo, jg, g);
     }
@@ -1336,6 +1337,7 @@ __global__ void __launch_bounds__(kThreads, 12) ccoll_decode_kernel(const __grid
     if (threadIdx.x == 0) {
       const uint32_t row0 = ((b.scatter ? 0u : jg.lo) + g * (uint32_t)kGroupValues) >> 5;
       tma_store_tile(&out_map, rows, row0, b.out_rank_stride ? (b.scatter ? y : dest) : 0u);
+      tma_store_wait();
     }
   } else {
     __syncthreads();
