@@ -284,7 +284,9 @@ static int allreduce_replay(const float* in, float* out, int P, size_t n, float 
         b.sum_out = out;
         b.sum_rank_stride = n;
       }
-      if (!launch_reduce(b, gx, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
+      // round k reads what round k-1 wrote and nothing else that a round writes: its grid may start (and fetch
+      // its local values) while round k-1 drains
+      if (!launch_reduce(b, gx, (uint32_t)P, s, /*behind_producer=*/true)) return CCOLL_ERR_CUDA;
       cur ^= 1;
     }
     if ((rc = check_launch()) != CCOLL_OK) return rc;
@@ -344,7 +346,7 @@ static int allreduce_replay(const float* in, float* out, int P, size_t n, float 
   d.P = P;
   d.skip_mode = 1;
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
-  if (Gc && !launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
+  if (Gc && !launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s, /*behind_producer=*/true)) return CCOLL_ERR_CUDA;
   return check_launch();
 }
 

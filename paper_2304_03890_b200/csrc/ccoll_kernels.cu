@@ -21,6 +21,7 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <utility>
 
 #include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; nothing links libcuda)
 
@@ -91,6 +92,11 @@ __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t* p) {
 __device__ __forceinline__ void st_relaxed_u64(uint64_t* p, uint64_t v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+// Programmatic dependent launch.  `grid_release` lets a grid launched behind this one (with the programmatic
+// attribute) start filling SM slots as soon as every CTA of this grid has begun; `grid_acquire` holds such a grid
+// until the grid before it has finished and its writes are visible.  Without the attribute both do nothing.
+__device__ __forceinline__ void grid_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_acquire() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ uint64_t pack_state(uint32_t epoch, uint32_t flag, uint32_t value) {
   return ((uint64_t)epoch << 32) | ((uint64_t)flag << 30) | (uint64_t)(value & kValueMask);
 }
@@ -1171,6 +1177,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __gri
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
+  grid_release();
   const JobGeom jg = job_geom(b.n, b.chunk_len, y);
   uint8_t* sout = b.sout + (uint64_t)y * b.s_stride;
   if (jg.G == 0) {
@@ -1203,9 +1210,11 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   Smem& sm = *reinterpret_cast<Smem*>(dyn_smem);
   uint8_t* rows = dyn_smem + kCtlBytes;
   const uint32_t g = blockIdx.x, y = blockIdx.y;
+  grid_release();
   const JobGeom jg = job_geom(b.n, b.chunk_len, y);
   uint8_t* sout = b.sout + (uint64_t)y * b.s_stride;
   if (jg.G == 0) {
+    grid_acquire();
     if (g == 0) write_empty_stream(b, y, sout);
     return;
   }
@@ -1227,6 +1236,9 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_reduce_kernel(const __grid_
   prefetch_group(local, jg, g + b.prefetch_distance);
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
 
+  // Everything above reads only this rank's own values, which no launch of a replay writes: in a replay this
+  // grid may get here while the round before it is still draining.  Its streams are read from here on.
+  grid_acquire();
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   StreamView sv;
@@ -1294,6 +1306,7 @@ __global__ void __launch_bounds__(kThreads, 12) ccoll_decode_kernel(const __grid
   const JobGeom jg = job_geom(b.n, b.chunk_len, y);
   if (g >= jg.G) return;
   const uint8_t* sin = b.sin + (uint64_t)y * b.s_stride;
+  grid_acquire();
   const uint64_t in_bytes = b.sin_bytes ? b.sin_bytes[y] : b.sin_bytes_host;
   const uint32_t dest = b.skip_mode == 4 ? (y + (uint32_t)b.rot) % (uint32_t)b.P : z;
   float* out = b.scatter ? b.out + (uint64_t)y * b.out_rank_stride : b.out + (uint64_t)dest * b.out_rank_stride + jg.lo;
@@ -1429,19 +1442,37 @@ bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cu
   ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemCompress, s>>>(b);
   return true;
 }
-bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
+// With `behind_producer` the grid is launched with the programmatic-serialisation attribute: its CTAs may take
+// the SM slots that the stream's previous grid (the producer of its input streams) leaves free while draining,
+// run up to their grid_acquire() and wait there.
+template <typename... Params, typename... Args>
+static void launch_grid(void (*kernel)(Params...), dim3 grid, int smem, cudaStream_t s, bool behind_producer, Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  std::memset(&attr, 0, sizeof(attr));
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = behind_producer ? 1u : 0u;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s, bool behind_producer) {
   if (!device_ready()) return false;
   EncodeBatch b = with_prefetch(b0, jobs);
   CUtensorMap x_map, sum_map;
   b.use_tma_in = rank_buffer_map(&x_map, b.x, b.n, b.x_rank_stride, b.P) ? 1 : 0;
   b.use_tma_sum = rank_buffer_map(&sum_map, b.sum_out, b.n, b.sum_rank_stride, b.P) ? 1 : 0;
-  if (b.op == 3)
-    ccoll_reduce_kernel<true><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b, x_map, sum_map);
-  else
-    ccoll_reduce_kernel<false><<<dim3(groups_x, jobs, 1), kThreads, kSmemBytes, s>>>(b, x_map, sum_map);
+  launch_grid(b.op == 3 ? ccoll_reduce_kernel<true> : ccoll_reduce_kernel<false>, dim3(groups_x, jobs, 1), kSmemBytes, s,
+              behind_producer, b, x_map, sum_map);
   return true;
 }
-bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s) {
+bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s,
+                   bool behind_producer) {
   if (!device_ready()) return false;
   DecodeBatch b = b0;
   // The output as a tensor of 128-byte rows: [32 values][rows of a destination][destinations].
@@ -1450,7 +1481,7 @@ bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint
   const uint64_t rows = (b.scatter ? b.chunk_len : b.n) / 32u;
   const uint64_t planes = b.out_rank_stride ? (b.scatter ? jobs : (b.skip_mode == 4 ? (uint32_t)b.P : ranks)) : 1u;
   b.use_tma = rows >= 128u && make_tile_map(&map, b.out, rows, planes, b.out_rank_stride * 4u, /*padded=*/false) ? 1 : 0;
-  ccoll_decode_kernel<<<dim3(groups_x, jobs, ranks), kThreads, kSmemDecode, s>>>(b, map);
+  launch_grid(ccoll_decode_kernel, dim3(groups_x, jobs, ranks), kSmemDecode, s, behind_producer, b, map);
   return true;
 }
 

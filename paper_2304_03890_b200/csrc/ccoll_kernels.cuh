@@ -90,7 +90,10 @@ constexpr uint32_t state_words(uint32_t tiles) { return tiles + (tiles + 31u) / 
 
 // Each returns false if the device could not be set up (the launch was not attempted).
 bool launch_compress(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
-bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s);
-bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s);
+// behind_producer: the stream's previous launch is the one that writes this launch's input streams (a replay's
+// rounds); the grid may then start while that launch drains and waits for it inside the kernel.
+bool launch_reduce(const EncodeBatch& b, uint32_t groups_x, uint32_t jobs, cudaStream_t s, bool behind_producer = false);
+bool launch_decode(const DecodeBatch& b, uint32_t groups_x, uint32_t jobs, uint32_t ranks, cudaStream_t s,
+                   bool behind_producer = false);
 
 }  // namespace ccoll
