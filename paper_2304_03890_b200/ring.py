@@ -18,8 +18,15 @@ Schedule on rank r of P (chunk c = values [c*C, (c+1)*C), C = ccoll_chunk_len):
                  owns chunk r+1)
   allgather      P-1 hops: forward the received stream unchanged, decompress a copy; the owner never
                  decompresses its own chunk.
-The decompression of hop h is queued on the device while the transfer of hop h+1 is already posted, which is
-the device-side counterpart of the overlap the paper obtains by polling (Sec. III-E).
+
+Overlap (Sec. III-E: the paper hides compression behind communication by polling between pieces of work).
+Here a chunk is cut into `segments` pieces on block boundaries, each a stream of its own, and the codec's
+operations are queued without waiting for them: while the device reduces and recompresses piece s of a round,
+the host is already exchanging piece s+1, and a piece's length is waited for only when it is about to be
+sent, one round later.  On a GPU the transfers are issued on a side stream, so that reading a length or
+staging a stream waits for that transfer alone and not for the kernels queued behind it.  The codec works
+block by block (Sec. III-D), so cutting on block boundaries leaves every decoded value unchanged: the result
+equals the unsegmented ring's (and the replay's) bit for bit; only the framing bytes on the wire grow.
 """
 import torch
 import torch.distributed as dist
@@ -27,29 +34,73 @@ import torch.distributed as dist
 from . import binding as B
 
 
+class Ready:
+    """A stream that is already complete (codecs that compute synchronously return these)."""
+
+    def __init__(self, stream):
+        self._stream = stream
+
+    def stream(self):
+        return self._stream
+
+
+class _Pending:
+    """A stream whose kernel is queued: its length reaches the host through a pinned word and an event."""
+
+    def __init__(self, buf, host_len, event, keep):
+        self.buf, self.host_len, self.event, self.keep = buf, host_len, event, keep
+
+    def stream(self):
+        self.event.synchronize()
+        return self.buf[: int(self.host_len[0])]
+
+
 class GpuCodec:
-    """The three device operations of the ring, through the C ABI."""
+    """The three device operations of the ring, through the C ABI, queued on the current CUDA stream."""
+
+    _SLOTS = 512  # lengths in flight at most (two per segment are)
 
     def __init__(self, eb, op=B.SUM, block_len=B.BLOCK_LEN):
         self.eb, self.op, self.block_len = float(eb), op, block_len
+        self._host = torch.zeros(self._SLOTS, dtype=torch.int64).pin_memory()
+        self._slot = 0
+
+    def prepare(self, longest):
+        """Called once before anything is queued: the workspace must not change while kernels are in flight."""
+        B.ensure_workspace(longest)
 
     def empty_stream(self, nbytes, like):
         return torch.empty(nbytes, dtype=torch.uint8, device=like.device)
 
-    def compress(self, x):
-        return B.compress(x, self.eb, self.block_len)
+    def _queued(self, n, device, launch):
+        out = torch.empty(B.ccoll_compress_bound(n, self.block_len), dtype=torch.uint8, device=device)
+        nbytes = torch.zeros(1, dtype=torch.int64, device=device)
+        launch(out, nbytes)
+        host_len = self._host[self._slot: self._slot + 1]
+        self._slot = (self._slot + 1) % self._SLOTS
+        host_len.copy_(nbytes, non_blocking=True)
+        event = torch.cuda.Event()
+        event.record()
+        return _Pending(out, host_len, event, (nbytes,))
 
-    def reduce_step(self, stream, local, want_result):
-        if want_result:
-            return B.reduce_step(stream, local, self.eb, want_sum=True, block_len=self.block_len, op=self.op)
-        return B.reduce_step(stream, local, self.eb, block_len=self.block_len, op=self.op), None
+    def compress(self, x):
+        return self._queued(x.numel(), x.device, lambda out, nb: B.ccoll_compress(x, self.eb, out, nb, self.block_len))
+
+    def reduce_step(self, stream, local, result_out):
+        return self._queued(local.numel(), local.device, lambda out, nb: B.ccoll_reduce_step_op(
+            stream, stream.numel(), local, self.eb, self.op, out, nb, result_out, self.block_len))
 
     def decompress(self, stream, n, out):
-        B.ensure_workspace(n)
         B.ccoll_decompress(stream, stream.numel(), n, out, self.block_len)
 
+    def finish(self):
+        """Waits for everything queued and raises if a kernel reported an error."""
+        status = B.ccoll_get_status()
+        if status != B.OK:
+            raise B.CcollError(status, "ring (device)")
 
-def _exchange(send_buf, like, codec, dst, src, group):
+
+def _exchange_here(send_buf, like, codec, dst, src, group):
     """Send `send_buf` (a uint8 stream) to dst and receive the neighbour's stream from src: lengths first."""
     # gloo carries host memory only: a device stream is then staged through the host (NCCL takes it as it is)
     staged = send_buf.is_cuda and dist.get_backend(group) == "gloo"
@@ -66,7 +117,30 @@ def _exchange(send_buf, like, codec, dst, src, group):
     return wire_in.to(send_buf.device) if staged else wire_in
 
 
-def c_allreduce(x, codec, group=None):
+def _exchange(send_buf, like, codec, dst, src, group, side):
+    """The exchange, on the side stream when there is one; the compute stream then waits for the received bytes."""
+    if side is None:
+        return _exchange_here(send_buf, like, codec, dst, src, group)
+    main = torch.cuda.current_stream()
+    with torch.cuda.stream(side):
+        send_buf.record_stream(side)   # allocated on the compute stream, read here
+        incoming = _exchange_here(send_buf, like, codec, dst, src, group)
+        incoming.record_stream(main)   # allocated here, read by kernels on the compute stream
+    main.wait_stream(side)
+    return incoming
+
+
+def segment_bounds(C, segments, block_len=B.BLOCK_LEN):
+    """Cuts [0, C) into at most `segments` pieces on block boundaries (on group boundaries, 32 blocks, where
+    the pieces are long enough): list of (lo, hi)."""
+    segments = max(1, int(segments))
+    unit = 32 * block_len if C >= segments * 32 * block_len else block_len
+    per = -(-C // segments)
+    per = max(unit, -(-per // unit) * unit)
+    return [(lo, min(lo + per, C)) for lo in range(0, max(C, 1), per)]
+
+
+def c_allreduce(x, codec, group=None, segments=1):
     """All-reduce of the 1-D fp32 tensor x over the ranks of `group`; returns (result, bytes this rank sent)."""
     P = dist.get_world_size(group)
     r = dist.get_rank(group)
@@ -79,24 +153,35 @@ def c_allreduce(x, codec, group=None):
     right, left = (r + 1) % P, (r - 1) % P
     if group is not None:
         right, left = dist.get_global_rank(group, right), dist.get_global_rank(group, left)
+    segs = segment_bounds(C, segments, codec.block_len)
+    side = torch.cuda.Stream(device=x.device) if x.is_cuda else None
 
-    def chunk(t, c):
-        return t[min(c * C, n): min((c + 1) * C, n)]
+    def piece(t, c, sg):
+        return t[min(c * C + sg[0], n): min(c * C + sg[1], n)]
 
+    if hasattr(codec, "prepare"):
+        codec.prepare(segs[0][1] - segs[0][0])
     sent = 0
-    cur = codec.compress(chunk(x, r))                      # round 0
-    for k in range(1, P):
-        sent += cur.numel()
-        incoming = _exchange(cur, x, codec, right, left, group)
-        c = (r - k) % P
-        cur, result = codec.reduce_step(incoming, chunk(x, c), want_result=(k == P - 1))
     owned = (r + 1) % P
-    chunk(out, owned).copy_(result)                        # the owner keeps the uncompressed result
+    cur = [codec.compress(piece(x, r, sg)) for sg in segs]        # round 0, all pieces queued
+    for k in range(1, P):
+        c = (r - k) % P
+        for i, sg in enumerate(segs):
+            mine = cur[i].stream()                                 # waits for this piece's kernel only
+            sent += mine.numel()
+            incoming = _exchange(mine, x, codec, right, left, group, side)
+            # the owner's round leaves the uncompressed result where it belongs
+            keep = piece(out, c, sg) if k == P - 1 else None
+            cur[i] = codec.reduce_step(incoming, piece(x, c, sg), keep if keep is not None and keep.numel() else None)
+    cur = [p.stream() for p in cur]
     for h in range(1, P):
-        sent += cur.numel()
-        cur = _exchange(cur, x, codec, right, left, group)  # forwarded unchanged on the next hop
         c = (owned - h) % P
-        dst = chunk(out, c)
-        if dst.numel():
-            codec.decompress(cur, dst.numel(), dst)
+        for i, sg in enumerate(segs):
+            sent += cur[i].numel()
+            cur[i] = _exchange(cur[i], x, codec, right, left, group, side)  # forwarded unchanged on the next hop
+            dst = piece(out, c, sg)
+            if dst.numel():
+                codec.decompress(cur[i], dst.numel(), dst)
+    if hasattr(codec, "finish"):
+        codec.finish()
     return out, sent

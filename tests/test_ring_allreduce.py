@@ -34,13 +34,15 @@ class OracleCodec:
         return torch.empty(nbytes, dtype=torch.uint8)
 
     def compress(self, x):
-        return torch.from_numpy(self.ccz.compress(x.numpy(), self.eb).copy())
+        from paper_2304_03890_b200.ring import Ready
+        return Ready(torch.from_numpy(self.ccz.compress(x.numpy(), self.eb).copy()))
 
-    def reduce_step(self, stream, local, want_result):
-        if want_result:
-            s, tot = self.ccz.reduce_step(stream.numpy(), local.numpy(), self.eb, want_sum=True, op=self.op)
-            return torch.from_numpy(s.copy()), torch.from_numpy(tot.copy())
-        return torch.from_numpy(self.ccz.reduce_step(stream.numpy(), local.numpy(), self.eb, op=self.op).copy()), None
+    def reduce_step(self, stream, local, result_out):
+        from paper_2304_03890_b200.ring import Ready
+        s, tot = self.ccz.reduce_step(stream.numpy(), local.numpy(), self.eb, want_sum=True, op=self.op)
+        if result_out is not None:
+            result_out.copy_(torch.from_numpy(tot.copy()))
+        return Ready(torch.from_numpy(s.copy()))
 
     def decompress(self, stream, n, out):
         out.copy_(torch.from_numpy(self.ccz.decompress(stream.numpy(), n).copy()))
@@ -52,7 +54,7 @@ def _inputs(world, n):
     return np.ascontiguousarray(c["x"].numpy()[:world, :n]), float(np.float32(c["eb"]))
 
 
-def _worker(rank, world, port, n, op, use_gpu, outdir):
+def _worker(rank, world, port, n, op, use_gpu, outdir, segments=1):
     sys.path.insert(0, ROOT)
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -64,16 +66,16 @@ def _worker(rank, world, port, n, op, use_gpu, outdir):
     else:
         codec = OracleCodec(eb, op)
         x = torch.from_numpy(xs[rank].copy())
-    out, sent = ring.c_allreduce(x, codec)
+    out, sent = ring.c_allreduce(x, codec, segments=segments)
     torch.save({"out": out.cpu(), "sent": sent}, os.path.join(outdir, f"r{rank}.pt"))
     dist.barrier()
     dist.destroy_process_group()
 
 
-def _run_and_check(tmp_path, world, n, op, use_gpu):
+def _run_and_check(tmp_path, world, n, op, use_gpu, segments=1):
     from oracle import ccz
     port = _free_port()
-    mp.spawn(_worker, args=(world, port, n, op, use_gpu, str(tmp_path)), nprocs=world, join=True)
+    mp.spawn(_worker, args=(world, port, n, op, use_gpu, str(tmp_path), segments), nprocs=world, join=True)
     xs, eb = _inputs(world, n)
     ref, ref_moved = ccz.allreduce_sim(xs, eb, op=op)
     sent = 0
@@ -81,7 +83,8 @@ def _run_and_check(tmp_path, world, n, op, use_gpu):
         got = torch.load(os.path.join(str(tmp_path), f"r{r}.pt"))
         assert got["out"].numpy().tobytes() == ref[r].tobytes(), f"rank {r}"
         sent += got["sent"]
-    assert sent == ref_moved
+    # one stream per chunk moves exactly the replay's bytes; cut into pieces, every piece adds its own frame
+    assert sent == ref_moved if segments == 1 else sent > ref_moved
 
 
 @pytest.mark.parametrize("world,n", [(2, 5000), (3, 128 * 37 + 5), (4, 24 * 24 * 32)])
@@ -93,7 +96,25 @@ def test_ring_max_on_cpu_ranks(tmp_path):
     _run_and_check(tmp_path, 3, 4096 * 2 + 77, 1, use_gpu=False)
 
 
+@pytest.mark.parametrize("world,n,segments", [(2, 5000, 3), (3, 24 * 24 * 32, 4), (4, 128 * 37 + 5, 2)])
+def test_ring_in_pieces_gives_the_same_values(tmp_path, world, n, segments):
+    """Chunks cut on block boundaries and pipelined piece by piece: the block-wise codec (Sec. III-D) decodes
+    every value as before, so each rank still holds its row of the unsegmented replay."""
+    _run_and_check(tmp_path, world, n, 0, use_gpu=False, segments=segments)
+
+
+def test_segment_bounds_cover_the_chunk_on_block_boundaries():
+    from paper_2304_03890_b200.ring import segment_bounds
+    for C, S in [(1, 1), (128, 4), (4608, 4), (4096 * 64, 8), (4096 * 64 + 128, 8), (1000064, 7), (128 * 5, 16)]:
+        b = segment_bounds(C, S)
+        assert b[0][0] == 0 and b[-1][1] == C and len(b) <= S
+        assert all(lo % 128 == 0 and hi > lo for lo, hi in b)
+        assert all(b[i][1] == b[i + 1][0] for i in range(len(b) - 1))
+        if C >= S * 4096:
+            assert all(lo % 4096 == 0 for lo, _ in b)
+
+
 @pytest.mark.gpu
-@pytest.mark.parametrize("world,n", [(2, 5000), (3, 24 * 24 * 32)])
-def test_ring_with_the_device_codec(tmp_path, world, n):
-    _run_and_check(tmp_path, world, n, 0, use_gpu=True)
+@pytest.mark.parametrize("world,n,segments", [(2, 5000, 1), (3, 24 * 24 * 32, 1), (2, 24 * 24 * 32 - 77, 3), (3, 24 * 24 * 32, 4)])
+def test_ring_with_the_device_codec(tmp_path, world, n, segments):
+    _run_and_check(tmp_path, world, n, 0, use_gpu=True, segments=segments)
