@@ -458,3 +458,56 @@ def test_seeded_fuzz_against_the_oracle():
         r_got, s_got = B.reduce_step(got, dev(y), eb, want_sum=True)
         assert np.array_equal(r_got.cpu().numpy(), r_ref), (case, n, eb)
         assert s_got.cpu().numpy().tobytes() == s_ref.tobytes(), (case, n, eb)
+
+
+def test_seeded_sweep_over_many_tiles_with_repeated_launches():
+    """Seeded cases long enough to span many groups and several 32-group size sums (20 k to 3 M values), each
+    launched more than once: the place of a group in its stream is found from the other groups' sizes while
+    they run, so a dependence on launch order would show as streams that differ from the oracle's or from one
+    another.  Streams, decoded values, one fused round (Sum / Max / Min) and, on every fourth case, a replay
+    with a random rank count and reduction must equal the oracle's bit for bit."""
+    rng = np.random.default_rng(23040389)
+    for case in range(48):
+        n = int(rng.choice([rng.integers(20000, 140000), rng.integers(140000, 600000), rng.integers(600000, 3000000)]))
+        t = np.arange(n, dtype=np.float64)
+        kind = case % 4
+        if kind == 0:
+            x = np.sin(t * rng.uniform(1e-4, 0.3)) * rng.uniform(0.1, 1e3)
+        elif kind == 1:
+            x = np.cumsum(rng.standard_normal(n)) * 10.0 ** rng.uniform(-3, 3)
+        elif kind == 2:
+            x = np.repeat(rng.standard_normal(n // 997 + 1), 997)[:n] + (rng.random(n) < 0.003) * rng.standard_normal(n)
+        else:
+            x = np.where((t // rng.integers(200, 5000)) % 2 == 0, np.sin(t * 1e-3) * 100, rng.uniform(-5, 5))
+        x = x.astype(np.float32)
+        if case % 6 == 0:
+            idx = rng.integers(0, n, size=3)
+            x[idx[0]], x[idx[1]], x[idx[2]] = np.nan, np.inf, -np.inf
+        finite = x[np.isfinite(x)]
+        eb = float(np.float32(max(float(finite.max() - finite.min()), 1e-30) * 10.0 ** rng.uniform(-6, -1)))
+        ref = ccz.compress(x, eb)
+        dx = dev(x)
+        for rep in range(2):
+            got = B.compress(dx, eb)
+            assert np.array_equal(got.cpu().numpy(), ref), (case, n, eb, rep)
+        assert B.decompress(got, n).cpu().numpy().tobytes() == ccz.decompress(ref, n).tobytes(), (case, n, eb)
+        y = np.roll(x, 13).copy()
+        y[~np.isfinite(y)] = 1.0
+        op = int(rng.integers(0, 3))
+        r_ref, s_ref = ccz.reduce_step(ref, y, eb, want_sum=True, op=op)
+        dy = dev(y)
+        for rep in range(2):
+            r_got, s_got = B.reduce_step(got, dy, eb, want_sum=True, op=op)
+            assert np.array_equal(r_got.cpu().numpy(), r_ref), (case, n, eb, op, rep)
+            assert s_got.cpu().numpy().tobytes() == s_ref.tobytes(), (case, n, eb, op, rep)
+        if case % 4 == 0:
+            P = int(rng.integers(2, 17))
+            m = (n // P) // 4 * 4
+            xs = np.stack([np.roll(x, 101 * r)[:m] for r in range(P)]).copy()
+            xs[~np.isfinite(xs)] = 0.5
+            op = int(rng.integers(0, 4))
+            o_ref, m_ref = ccz.allreduce_sim(xs, eb, op=op)
+            dxs = dev(xs)
+            for rep in range(2):
+                o_got, m_got = B.allreduce_sim(dxs, eb, op=op)
+                assert o_got.cpu().numpy().tobytes() == o_ref.tobytes() and m_got == m_ref, (case, P, m, eb, op, rep)
