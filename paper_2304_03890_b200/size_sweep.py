@@ -7,6 +7,12 @@ For every size (a smooth 3-D field of that many bytes, the recipe of the 512x512
 bound it prints the compression ratio, the device time of compress, decompress and the replayed all-reduce
 over P virtual ranks (the buffer viewed as P rank buffers), and PSNR / NRMSE / largest error of the round trip.
 Timing runs through the C ABI; the quality figures are plain reductions over the decoded buffer.
+
+    python -m paper_2304_03890_b200.size_sweep --small
+
+times the 2^20-value case (four sines plus noise, 4 MiB: it fits the L2 cache many times over) as CUDA graphs
+of 64 launches and prints median and minimum per launch of compress, decompress and the fused round twice: on one buffer
+(L2-hot) and rotating over 64 copies of it (256 MiB of inputs and as many streams: HBM-cold).
 """
 import argparse
 import math
@@ -38,12 +44,67 @@ def quality(x, y):
     return psnr, rmse / rng, float(d.abs().max())
 
 
+def per_launch(fn, copies, launches=64, replays=20):
+    """Device time per launch in us, (median, min) over replays of a CUDA graph of `launches` launches: a call
+    of this size is shorter than the host's work to issue it, so launches timed one by one would measure the
+    host."""
+    for i in range(copies):
+        fn(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(launches):
+            fn(i % copies)
+    graph.replay()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(replays)]
+    for a, b in ev:
+        a.record()
+        graph.replay()
+        b.record()
+    torch.cuda.synchronize()
+    t = sorted(a.elapsed_time(b) * 1e3 / launches for a, b in ev)
+    return t[len(t) // 2], t[0]
+
+
+def small():
+    cfg = fields.config1(device="cuda")
+    x, eb = cfg["x"].reshape(-1), float(cfg["eb"])
+    n = x.numel()
+    copies = 64
+    xs = x.repeat(copies, 1).contiguous()
+    B.ensure_workspace(n)
+    cap = (B.ccoll_compress_bound(n) + 255) // 256 * 256
+    ss = torch.empty((copies, cap), dtype=torch.uint8, device="cuda")
+    rs = torch.empty_like(ss)
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    dec = torch.empty_like(xs)
+    for i in range(copies):
+        B.ccoll_compress(xs[i], eb, ss[i], nb)
+    nbytes = int(nb.item())
+    print(f"n = {n} values ({4 * n / 2**20:.0f} MiB), eb = {eb:.4g}, CR = {4 * n / nbytes:.2f}")
+    print("call        buffers  median_us  min_us  GB/s_of_fp32_at_median")
+    calls = {
+        "compress": lambda i: B.ccoll_compress(xs[i], eb, ss[i], nb),
+        "decompress": lambda i: B.ccoll_decompress(ss[i], nbytes, n, dec[i]),
+        "reduce_step": lambda i: B.ccoll_reduce_step(ss[i], nbytes, xs[i], eb, rs[i], nb),
+    }
+    for name, fn in calls.items():
+        for label, c in (("1 (L2-hot)", 1), (f"{copies} (HBM-cold)", copies)):
+            med, mn = per_launch(fn, c)
+            print(f"{name:11s} {label:14s} {med:8.2f} {mn:8.2f} {4 * n / med / 1e3:8.0f}")
+    assert B.ccoll_get_status() == B.OK
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sizes-mb", default="278,478,678")
     ap.add_argument("--rel-eb", default="1e-2,1e-3,1e-4")
     ap.add_argument("--P", type=int, default=8)
+    ap.add_argument("--small", action="store_true", help="the 2^20-value case, L2-hot and HBM-cold, per launch")
     args = ap.parse_args()
+    if args.small:
+        small()
+        return
     P = args.P
     print("size_MB rel_eb CR compress_ms GB/s decompress_ms GB/s allreduce_ms PSNR_dB NRMSE max_err/eb")
     for mb in (float(v) for v in args.sizes_mb.split(",")):
