@@ -15,7 +15,9 @@
  *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".  The library
  *     allocates nothing; scratch comes from the workspace the caller registers with ccoll_set_workspace.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is enqueued
- *     on it and the call returns without waiting.
+ *     on it and the call returns without waiting.  Apart from ccoll_get_status (which waits for the stream)
+ *     and ccoll_set_workspace no entry point makes a synchronising call, so a sequence of calls can be
+ *     captured into a CUDA graph.
  *   - Return value: a ccoll_status_t for errors the host can see (bad argument, missing workspace, CUDA
  *     launch failure).  Errors only the GPU can see (corrupt stream, capacity, look-back time-out) go to a
  *     sticky status word in the workspace; read and clear it with ccoll_get_status.

@@ -1436,8 +1436,23 @@ static bool rank_buffer_map(CUtensorMap* map, const float* base, uint64_t n, uin
   return base && n / 32u >= 128u &&
          make_tile_map(map, base, n / 32u, rank_stride ? (uint64_t)P : 1u, rank_stride * 4u, /*padded=*/true);
 }
+// A launch that is being captured into a CUDA graph will run again with the epoch it was captured with, and
+// would then take its own size words of the previous replay for fresh ones.  Such a launch gets a memset node
+// in front of it that clears its size words (epoch 0 is never used), so every replay starts from "not written".
+static bool is_capturing(cudaStream_t s) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &st) != cudaSuccess) {
+    cudaGetLastError();  // e.g. the legacy stream while another stream captures: not a capture of this launch
+    return false;
+  }
+  return st == cudaStreamCaptureStatusActive;
+}
+static bool clear_sizes(const EncodeBatch& b, uint32_t jobs, cudaStream_t s) {
+  const size_t words = (size_t)jobs * b.state_stride;
+  return words == 0 || cudaMemsetAsync(b.tile_state, 0, words * sizeof(uint64_t), s) == cudaSuccess;
+}
 bool launch_compress(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s) {
-  if (!device_ready()) return false;
+  if (!device_ready() || (is_capturing(s) && !clear_sizes(b0, jobs, s))) return false;
   const EncodeBatch b = with_prefetch(b0, jobs);
   ccoll_compress_kernel<<<dim3(groups_x, jobs, 1), kThreads, kSmemCompress, s>>>(b);
   return true;
@@ -1463,6 +1478,10 @@ static void launch_grid(void (*kernel)(Params...), dim3 grid, int smem, cudaStre
 }
 bool launch_reduce(const EncodeBatch& b0, uint32_t groups_x, uint32_t jobs, cudaStream_t s, bool behind_producer) {
   if (!device_ready()) return false;
+  if (is_capturing(s)) {  // (captured launches are plain ones: the memset node sits between this grid and its producer)
+    if (!clear_sizes(b0, jobs, s)) return false;
+    behind_producer = false;
+  }
   EncodeBatch b = with_prefetch(b0, jobs);
   CUtensorMap x_map, sum_map;
   b.use_tma_in = rank_buffer_map(&x_map, b.x, b.n, b.x_rank_stride, b.P) ? 1 : 0;
@@ -1481,7 +1500,7 @@ bool launch_decode(const DecodeBatch& b0, uint32_t groups_x, uint32_t jobs, uint
   const uint64_t rows = (b.scatter ? b.chunk_len : b.n) / 32u;
   const uint64_t planes = b.out_rank_stride ? (b.scatter ? jobs : (b.skip_mode == 4 ? (uint32_t)b.P : ranks)) : 1u;
   b.use_tma = rows >= 128u && make_tile_map(&map, b.out, rows, planes, b.out_rank_stride * 4u, /*padded=*/false) ? 1 : 0;
-  launch_grid(ccoll_decode_kernel, dim3(groups_x, jobs, ranks), kSmemDecode, s, behind_producer, b, map);
+  launch_grid(ccoll_decode_kernel, dim3(groups_x, jobs, ranks), kSmemDecode, s, behind_producer && !is_capturing(s), b, map);
   return true;
 }
 

@@ -511,3 +511,86 @@ def test_seeded_sweep_over_many_tiles_with_repeated_launches():
             for rep in range(2):
                 o_got, m_got = B.allreduce_sim(dxs, eb, op=op)
                 assert o_got.cpu().numpy().tobytes() == o_ref.tobytes() and m_got == m_ref, (case, P, m, eb, op, rep)
+
+
+def test_calls_captured_into_a_cuda_graph():
+    """The entry points only enqueue work, so a sequence of them can be captured once and replayed: the
+    replays (on new input contents in the same buffers) must still equal the oracle bit for bit."""
+    P, m = 4, 4096 * 6 + 512
+    n = P * m
+    rng = np.random.default_rng(7)
+    eb = 1e-3
+    x = torch.zeros(n, device="cuda")
+    B.ensure_workspace(n, P)
+    s = torch.empty(B.ccoll_compress_bound(n), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    out = torch.empty((P, m), device="cuda")
+    moved = torch.zeros(1, dtype=torch.int64, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):  # first use of the kernels outside the capture
+        B.ccoll_compress(x, eb, s, nb)
+        B.ccoll_allreduce_sim(x.view(P, m), out, eb, moved)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.ccoll_compress(x, eb, s, nb)
+        B.ccoll_allreduce_sim(x.view(P, m), out, eb, moved)
+    for rep in range(3):
+        h = np.cumsum(rng.standard_normal(n)).astype(np.float32)
+        x.copy_(torch.from_numpy(h))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = ccz.compress(h, eb)
+        assert int(nb.item()) == ref.size and np.array_equal(s[: ref.size].cpu().numpy(), ref), rep
+        o_ref, m_ref = ccz.allreduce_sim(h.reshape(P, m), eb)
+        assert out.cpu().numpy().tobytes() == o_ref.tobytes() and int(moved.item()) == m_ref, rep
+    assert B.ccoll_get_status() == B.OK
+
+
+def test_a_graph_of_one_launch_replayed_on_changing_data():
+    """A captured launch runs again with the epoch it was captured with; its size words of the previous replay
+    must not be taken for fresh ones.  One compress and one fused round, each alone in its graph, replayed on
+    data whose group sizes change completely from replay to replay."""
+    n = 4096 * 300 + 77
+    eb = 1e-3
+    rng = np.random.default_rng(11)
+    x = torch.zeros(n, device="cuda")
+    B.ensure_workspace(n)
+    cap = B.ccoll_compress_bound(n)
+    s = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    r = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    nr = torch.zeros(1, dtype=torch.int64, device="cuda")
+    tot = torch.empty(n, device="cuda")
+    B.ccoll_compress(x, eb, s, nb)
+    first = int(nb.item())
+    B.ccoll_reduce_step(s, first, x, eb, r, nr, tot)
+    torch.cuda.synchronize()
+    g_c, g_r = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_c):
+        B.ccoll_compress(x, eb, s, nb)
+    inputs = [np.zeros(n, np.float32),                                        # all constant: the smallest stream
+              (rng.standard_normal(n) * 50).astype(np.float32),              # noise: large records
+              np.sin(np.arange(n) * 1e-3).astype(np.float32),                # smooth: small records
+              np.where(np.arange(n) % 8192 < 4096, 0.0, rng.standard_normal(n)).astype(np.float32)]
+    for rep, h in enumerate(inputs):
+        x.copy_(torch.from_numpy(h))
+        g_c.replay()
+        torch.cuda.synchronize()
+        ref = ccz.compress(h, eb)
+        assert int(nb.item()) == ref.size and np.array_equal(s[: ref.size].cpu().numpy(), ref), rep
+    # the fused round: a fixed incoming stream (the last one above), changing local values
+    in_bytes = int(nb.item())
+    incoming = s[:in_bytes].cpu().numpy().copy()
+    with torch.cuda.graph(g_r):
+        B.ccoll_reduce_step(s, in_bytes, x, eb, r, nr, tot)
+    for rep, h in enumerate(inputs):
+        x.copy_(torch.from_numpy(h))
+        g_r.replay()
+        torch.cuda.synchronize()
+        r_ref, t_ref = ccz.reduce_step(incoming, h, eb, want_sum=True)
+        assert int(nr.item()) == r_ref.size and np.array_equal(r[: r_ref.size].cpu().numpy(), r_ref), rep
+        assert tot.cpu().numpy().tobytes() == t_ref.tobytes(), rep
+    assert B.ccoll_get_status() == B.OK
