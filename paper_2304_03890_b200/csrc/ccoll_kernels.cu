@@ -335,6 +335,38 @@ __device__ __forceinline__ void load_rows_padded(uint8_t* rows, const float* x, 
     dst[r * kRoundStride] = v;
   }
 }
+// The same with every warp loading its own 32 rows (4 KB of the group): in round r lane l moves the float4
+// number 256 w + 32 r + l, piece (l & 7) of row 32 w + 4 r + l / 8.  A warp then depends on its own loads only:
+// a __syncwarp is enough before its lanes read their rows.
+__device__ __forceinline__ void load_rows_padded_own(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t cnt = group_count(jg, g);
+  const float* src = x + (size_t)g * kGroupValues;
+  const uint32_t f0 = 256u * warp + lane;  // the thread's float4 of round 0
+  float4* dst = reinterpret_cast<float4*>(rows + (32u * warp + (lane >> 3)) * kPaddedRowBytes + 16u * (lane & 7u));
+  constexpr int kRoundStride = 4 * kPaddedRowBytes / 16;  // float4s between a thread's rounds (four rows)
+  if (cnt == (uint32_t)kGroupValues) {
+    float4 t[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t[r] = __ldcs(reinterpret_cast<const float4*>(src) + f0 + 32 * r);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) dst[r * kRoundStride] = t[r];
+    return;
+  }
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = f0 + 32u * (uint32_t)r;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (4u * f + 4u <= cnt) {
+      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
+    } else {
+      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
+    }
+    dst[r * kRoundStride] = v;
+  }
+}
 // A swizzled tile without the TMA unit (a group that is not complete, or no tensor map): coalesced 128-bit
 // streaming stores, bounds watched; thread tid moves the float4 number r*128 + tid in round r, which is piece
 // (tid & 7) of row 16 r + tid / 8.  A __syncthreads must separate it from the writes of the rows.
@@ -1192,11 +1224,11 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __gri
   // (A TMA tile load into these rows was measured too: 78 us against 71 us.  Nothing else can run in this CTA
   // until its values are there, and the one bulk request comes back later than eight rounds of plain loads; in
   // the fused round the same tile load hides behind the staging of the payload and wins.)
-  load_rows_padded(rows, x, jg, g);
+  load_rows_padded_own(rows, x, jg, g);
   prefetch_group(x, jg, g + b.prefetch_distance);
-  zero_image(sm.img);
+  zero_image(sm.img);  // (this and the two words below are first used behind the barrier inside encode_group)
   if (threadIdx.x == 0) sm.prefix = 0u, sm.fail = 0u;
-  __syncthreads();
+  __syncwarp();  // a warp reads only rows that it loaded itself
   if (tail) pad_ragged<PaddedRow>(rows, lg);
   float mx, mn;
   lane_minmax(make_row<PaddedRow>(rows, threadIdx.x), mx, mn);
