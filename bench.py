@@ -338,45 +338,62 @@ def main():
 
     # The copies run on streams of their own, ordered against the calls by events: x2 goes up while compress and
     # decompress run, and every result starts down as soon as its call has finished (PCIe carries both ways).
-    s_in, s_out, cur = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
-    ev = [torch.cuda.Event() for _ in range(8)]
+    # Steps alternate between two sets of device buffers, as a caller that feeds one buffer after another would
+    # run them: while the results of a step go down, the inputs of the next one come up and its calls run.  A
+    # set is written again only when the step that used it before has been read out.
+    s_in, s_out, s_len, cur = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    first = dict(x=x, x2=x2, s1=s1, nb1=nb1, dec=dec, s2=s2, nb2=nb2, ssum=ssum, ar=ar_out)
+    sets = [first, {k: torch.empty_like(v) for k, v in first.items()}]
+    for d in sets:
+        d["ev"] = [torch.cuda.Event() for _ in range(6)]
+        d["calls_done"], d["read_out"], d["used"] = torch.cuda.Event(), torch.cuda.Event(), False
+    step_no = 0
 
     def e2e_step():
-        nonlocal d2h
-        s_in.wait_stream(cur)      # the previous step's calls are done with x and x2
-        s_out.wait_stream(cur)
+        nonlocal d2h, step_no
+        d = sets[step_no % 2]
+        step_no += 1
+        ev = d["ev"]
         with torch.cuda.stream(s_in):
-            x.copy_(hx, non_blocking=True)
+            if d["used"]:
+                s_in.wait_event(d["calls_done"])   # the calls that read these inputs two steps ago
+            d["x"].copy_(hx, non_blocking=True)
             ev[0].record(s_in)
-            x2.copy_(hx2, non_blocking=True)
+            d["x2"].copy_(hx2, non_blocking=True)
             ev[1].record(s_in)
+        if d["used"]:
+            cur.wait_event(d["read_out"])          # the results these calls overwrite have gone down
         cur.wait_event(ev[0])
-        B.ccoll_compress(x, eb, s1, nb1)
+        B.ccoll_compress(d["x"], eb, d["s1"], d["nb1"])
         ev[2].record(cur)
-        B.ccoll_decompress(s1, in_bytes, n, dec)
+        B.ccoll_decompress(d["s1"], in_bytes, n, d["dec"])
         ev[3].record(cur)
         cur.wait_event(ev[1])
-        B.ccoll_reduce_step(s1, in_bytes, x2, eb, s2, nb2, ssum)
+        B.ccoll_reduce_step(d["s1"], in_bytes, d["x2"], eb, d["s2"], d["nb2"], d["ssum"])
         ev[4].record(cur)
-        B.ccoll_allreduce_sim(xr, ar_out.view(P, n // P), eb, moved)
+        B.ccoll_allreduce_sim(d["x"].view(P, n // P), d["ar"].view(P, n // P), eb, moved)
         ev[5].record(cur)
-        B.ccoll_bcast_sim(x, sc_out, C, P, eb, B.SCATTER, cb)
+        B.ccoll_bcast_sim(d["x"], sc_out, C, P, eb, B.SCATTER, cb)
+        d["calls_done"].record(cur)
+        with torch.cuda.stream(s_len):             # the stream's length, on a stream that carries nothing else
+            s_len.wait_event(ev[2])
+            h_nb.copy_(d["nb1"], non_blocking=True)
+        s_len.synchronize()
+        sb = int(h_nb.item())
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev[2])
-            h_nb.copy_(nb1, non_blocking=True)
-            s_out.synchronize()
-            sb = int(h_nb.item())
-            h_s1[:sb].copy_(s1[:sb], non_blocking=True)
+            h_s1[:sb].copy_(d["s1"][:sb], non_blocking=True)
             s_out.wait_event(ev[3])
-            h_dec.copy_(dec, non_blocking=True)
+            h_dec.copy_(d["dec"], non_blocking=True)
             s_out.wait_event(ev[4])
-            h_sum.copy_(ssum, non_blocking=True)
+            h_sum.copy_(d["ssum"], non_blocking=True)
             s_out.wait_event(ev[5])
-            h_ar.copy_(ar_out, non_blocking=True)
-        s_out.synchronize()
-        cur.synchronize()
+            h_ar.copy_(d["ar"], non_blocking=True)
+            d["read_out"].record(s_out)
+        d["used"] = True
         d2h = sb + 3 * 4 * n + 8
 
+    e2e_step()
     e2e_step()
     sync_all()
     t0 = time.perf_counter()
