@@ -65,8 +65,11 @@ class GpuCodec:
         self._host = torch.zeros(self._SLOTS, dtype=torch.int64).pin_memory()
         self._slot = 0
 
-    def prepare(self, longest):
-        """Called once before anything is queued: the workspace must not change while kernels are in flight."""
+    def prepare(self, longest, in_flight):
+        """Called once before anything is queued: the workspace must not change while kernels are in flight,
+        and every stream whose length has not been read yet needs a pinned word of its own."""
+        if in_flight > self._SLOTS:
+            raise ValueError(f"at most {self._SLOTS // 2} segments")
         B.ensure_workspace(longest)
 
     def empty_stream(self, nbytes, like):
@@ -160,7 +163,7 @@ def c_allreduce(x, codec, group=None, segments=1):
         return t[min(c * C + sg[0], n): min(c * C + sg[1], n)]
 
     if hasattr(codec, "prepare"):
-        codec.prepare(segs[0][1] - segs[0][0])
+        codec.prepare(segs[0][1] - segs[0][0], 2 * len(segs))
     sent = 0
     owned = (r + 1) % P
     cur = [codec.compress(piece(x, r, sg)) for sg in segs]        # round 0, all pieces queued
