@@ -253,6 +253,7 @@ struct PaddedRow {
   __device__ __forceinline__ uint4 words4(uint32_t j) const { return *reinterpret_cast<const uint4*>(p + 16u * j); }
   __device__ __forceinline__ uint32_t word(uint32_t i) const { return *reinterpret_cast<const uint32_t*>(p + 4u * i); }
   __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const { *reinterpret_cast<uint32_t*>(p + 4u * i) = v; }
+  __device__ __forceinline__ uint32_t* word_ptr(uint32_t i) const { return reinterpret_cast<uint32_t*>(p + 4u * i); }
 };
 template <class RowT>
 __device__ __forceinline__ RowT make_row(uint8_t* rows, uint32_t t);
@@ -505,6 +506,7 @@ __device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t 
   uint32_t lo = 0u, hi = 0u, Tb = 0u;
   uint32_t clo = 0u, chi = 0u;
   const uint32_t rot = RowT::rot(threadIdx.x);  // staged word k goes to word rot + k of the row
+  uint32_t* wp = row.word_ptr(rot);             // where the next completed word goes
   auto put = [&](uint32_t q, uint32_t sa) {
     const uint32_t n = 32u - sa;
     const uint32_t t = __funnelshift_lc(0u, q, sa);  // the stored bits, at the top of the word
@@ -512,7 +514,7 @@ __device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t 
     hi = __funnelshift_lc(lo, hi, n);
     lo = __funnelshift_lc(t, lo, n);
     if ((Tn ^ Tb) & 32u)  // a word boundary was crossed (n <= 32: at most one)
-      row.set_word(rot + (Tn >> 5) - 1u, __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123));
+      *wp++ = __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123);
     Tb = Tn;
   };
   // the next quad is always read before the current one's words are stored: they may reach rot <= 3 words
