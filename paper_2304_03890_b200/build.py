@@ -9,7 +9,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SOURCES = [os.path.join(CSRC, f) for f in ("ccoll_kernels.cu", "ccoll_api.cu", "ccoll_noalloc.cu")]
-HEADERS = [os.path.join(CSRC, "ccoll_kernels.cuh"), os.path.join(os.path.dirname(HERE), "include", "ccoll.h")]
+HEADERS = [os.path.join(CSRC, f) for f in ("ccoll_kernels.cuh", "ccoll_device_common.cuh", "ccoll_encode.cuh",
+                                            "ccoll_decode.cuh")] + [os.path.join(os.path.dirname(HERE), "include", "ccoll.h")]
 LIB = os.path.join(HERE, "libccoll.so")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "--fmad=false",

@@ -1,0 +1,378 @@
+// ccoll_decode.cuh — the decoder of a group: validation of the stream's frame, staging of the payload, record
+// offsets, the predecessor chain across lanes and the value loop (which, in the fused round, reduces into the
+// lane's row instead of returning the values).  Included by ccoll_kernels.cu only, after ccoll_encode.cuh
+// (whose warp scans it uses).
+#pragma once
+#include "ccoll_encode.cuh"
+
+namespace ccoll {
+namespace {
+
+// ---------------------------------------------------------------------------------------------------
+// decode side
+// ---------------------------------------------------------------------------------------------------
+struct StreamView {
+  const uint32_t* words;  // the stream as 32-bit words
+  uint32_t G, base;       // groups, payload_base
+  uint32_t a, gw, map;    // first payload word of the group, its length in words, its bitmap
+  uint32_t pw;            // payload words of the whole stream
+};
+
+// Validate the header and the directory entries of group g.  Every thread of the CTA reads the same words
+// and reaches the same verdict.
+__device__ __forceinline__ bool open_group(const uint8_t* sin, uint64_t in_bytes, const JobGeom& jg, uint32_t g,
+                                           StreamView& sv) {
+  sv.words = reinterpret_cast<const uint32_t*>(sin);
+  sv.G = jg.G;
+  sv.base = payload_base(jg.G);
+  if (in_bytes < sv.base) return false;
+  const uint32_t* w = sv.words;
+  uint64_t n = (uint64_t)__ldg(w + 2) | ((uint64_t)__ldg(w + 3) << 32);
+  uint64_t total = (uint64_t)__ldg(w + 6) | ((uint64_t)__ldg(w + 7) << 32);
+  if (__ldg(w) != kMagic || __ldg(w + 1) != 0u || n != jg.len || __ldg(w + 4) != (uint32_t)kL) return false;
+  if (total > in_bytes || total < sv.base || ((total - sv.base) & 3u)) return false;
+  uint64_t pw = (total - sv.base) >> 2;  // payload words
+  uint32_t a = __ldg(w + 8 + g), e = __ldg(w + 8 + g + 1);
+  sv.map = __ldg(w + 8 + jg.G + 1 + g);
+  if (a > e || (uint64_t)e > pw || (e - a) * 4u > (uint32_t)kMaxGroupBytes) return false;
+  if (g == jg.G - 1 && (uint64_t)e != pw) return false;
+  uint32_t nblk = min((uint32_t)kGroupBlocks, jg.nb - g * kGroupBlocks);
+  if (nblk < 32u && (sv.map >> nblk) != 0u) return false;
+  sv.a = a;
+  sv.gw = e - a;
+  sv.pw = (uint32_t)pw;
+  return true;
+}
+
+// sum of the sixteen 2-bit fields of a word
+__device__ __forceinline__ uint32_t sum_fields(uint32_t w) {
+  return (uint32_t)__popc(w & 0x55555555u) + 2u * (uint32_t)__popc(w & 0xaaaaaaaau);
+}
+
+// One byte position of a lane's summary.  The lane's 32 lead codes sit in two words (values 0-15 in lo,
+// 16-31 in hi).  Values with lead <= KB store byte KB of the field (counted from its most significant
+// byte); the last such value is found with one leading-zero count, the stored bytes before it with two
+// population counts, and its byte is fetched from the image.
+struct SummaryIn {
+  uint32_t lo, hi, lo1, hi1;  // the codes, and the codes shifted right by one
+  uint32_t vlo, vhi;          // marker bit (even positions) of every valid value
+  uint32_t lead_lo;           // sum of the leads of values 0-15
+  uint32_t B, pos0;
+};
+template <int KB>
+__device__ __forceinline__ void summary_byte(const uint32_t* img, const SummaryIn& si, uint32_t& sval, uint32_t& smask) {
+  uint32_t ph, pl;  // markers of the values that store byte KB
+  if (KB == 0) {
+    ph = ~(si.hi | si.hi1) & si.vhi;
+    pl = ~(si.lo | si.lo1) & si.vlo;
+  } else if (KB == 1) {
+    ph = ~si.hi1 & si.vhi;
+    pl = ~si.lo1 & si.vlo;
+  } else if (KB == 2) {
+    ph = ~(si.hi & si.hi1) & si.vhi;
+    pl = ~(si.lo & si.lo1) & si.vlo;
+  } else {
+    ph = si.vhi;
+    pl = si.vlo;
+  }
+  if ((ph | pl) == 0u) return;
+  const bool up = ph != 0u;
+  const uint32_t pm = up ? ph : pl, w = up ? si.hi : si.lo;
+  const uint32_t i2 = 31u - (uint32_t)__clz((int)pm);  // bit position of the value's code = 2 * (its index in the half)
+  const uint32_t below = w & ((1u << i2) - 1u);        // codes of the values before it in this half
+  const uint32_t lead_sum = (up ? si.lead_lo : 0u) + sum_fields(below);
+  const uint32_t lead_i = (w >> i2) & 3u;
+  const uint32_t i = (i2 >> 1) + (up ? 16u : 0u);
+  const uint32_t byte = img_u8(img, si.pos0 + (si.B * i - lead_sum) + ((uint32_t)KB - lead_i));
+  const uint32_t shift = 8u * (si.B - 1u - (uint32_t)KB);
+  sval |= byte << shift;
+  smask |= 0xffu << shift;
+}
+
+// One quad of the general decode path: any field width, lossless blocks, ragged slices (nvq = valid values
+// of the quad).  Out of line on purpose (rare, and it keeps the kernels' hot code small).
+struct DecodeCursor {
+  uint32_t pos;   // image offset of the next stored byte
+  uint32_t prev;  // code of the previous value
+};
+__device__ __noinline__ float4 decode_quad_generic(const uint32_t* img, DecodeCursor& cur, uint32_t cb, uint32_t R,
+                                                   float mu, uint32_t nvq) {
+  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
+  uint32_t nb0 = B - (cb & 3u), nb1 = B - ((cb >> 2) & 3u), nb2 = B - ((cb >> 4) & 3u), nb3 = B - ((cb >> 6) & 3u);
+  if (nvq < 1u) nb0 = 0u;
+  if (nvq < 2u) nb1 = 0u;
+  if (nvq < 3u) nb2 = 0u;
+  if (nvq < 4u) nb3 = 0u;
+  // the quad's stored bytes as a little-endian 16-byte string
+  const uint32_t wi = cur.pos >> 2, z = 8u * (cur.pos & 3u);
+  const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3], A4 = img[wi + 4];
+  const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z),
+                 S3 = __funnelshift_r(A3, A4, z);
+  cur.pos += nb0 + nb1 + nb2 + nb3;
+  // peel the four values off the front of the string
+  const uint32_t c0 = 8u * nb0, c1 = 8u * nb1, c2 = 8u * nb2, c3 = 8u * nb3;
+  const uint32_t U0 = __funnelshift_rc(S0, S1, c0), U1 = __funnelshift_rc(S1, S2, c0), U2 = __funnelshift_rc(S2, S3, c0);
+  const uint32_t X0 = __funnelshift_rc(U0, U1, c1), X1 = __funnelshift_rc(U1, U2, c1);
+  const uint32_t r3 = __funnelshift_rc(X0, X1, c2);
+  // stored bytes as a right-aligned big-endian value; the bytes not stored come from the predecessor
+  const uint32_t v0 = __funnelshift_rc(__byte_perm(S0, 0u, 0x0123), 0u, 32u - c0);
+  const uint32_t v1 = __funnelshift_rc(__byte_perm(U0, 0u, 0x0123), 0u, 32u - c1);
+  const uint32_t v2 = __funnelshift_rc(__byte_perm(X0, 0u, 0x0123), 0u, 32u - c2);
+  const uint32_t v3 = __funnelshift_rc(__byte_perm(r3, 0u, 0x0123), 0u, 32u - c3);
+  const uint32_t q0 = v0 | (cur.prev & ~__funnelshift_rc(kFull, 0u, 32u - c0));
+  const uint32_t q1 = v1 | (q0 & ~__funnelshift_rc(kFull, 0u, 32u - c1));
+  const uint32_t q2 = v2 | (q1 & ~__funnelshift_rc(kFull, 0u, 32u - c2));
+  const uint32_t q3 = v3 | (q2 & ~__funnelshift_rc(kFull, 0u, 32u - c3));
+  cur.prev = q3;
+  if (R == 32u) return make_float4(__uint_as_float(q0), __uint_as_float(q1), __uint_as_float(q2), __uint_as_float(q3));
+  return make_float4(__fadd_rn(__uint_as_float(q0 << sh), mu), __fadd_rn(__uint_as_float(q1 << sh), mu),
+                     __fadd_rn(__uint_as_float(q2 << sh), mu), __fadd_rn(__uint_as_float(q3 << sh), mu));
+}
+
+// One reduction of the collective-computation framework (Sec. III-B): a = decoded value, b = local value.
+// Sum: one rounded add (a NaN result is the GPU's canonical 0x7FFFFFFF).  Max / Min: a pure selection, a if
+// it beats b or b is a NaN, else b.  kDivide (the owner's round of an Average, a kernel of its own so that the
+// division costs the other rounds nothing): the sum, then one correctly rounded division by the number of
+// ranks; a NaN quotient is made the same canonical NaN.
+template <bool kDivide>
+__device__ __forceinline__ float reduce_op(float a, float b, int op, float divisor) {
+  if (kDivide) {
+    const float q = __fdiv_rn(__fadd_rn(a, b), divisor);
+    return q != q ? __uint_as_float(0x7fffffffu) : q;
+  }
+  if (op == 0) return __fadd_rn(a, b);
+  if (op == 1) return (a > b || b != b) ? a : b;
+  return (a < b || b != b) ? a : b;
+}
+
+// Decode the lane's 32 values of group g into v[].  Returns false (for the whole CTA) on a corrupt group.
+// The group's payload must already be staged in sm.img (and visible).  nblk = blocks in the group.
+// kToSlice = false: the values are returned in v[] (fully unrolled loops).  kToSlice = true (fused reduce):
+// each decoded quad is REDUCED (op) with the quad of local values waiting in the lane's slice and the result is written
+// back there, and mx / mn receive the largest / smallest result of the lane (meaningless for a ragged slice);
+// the loops are then unrolled only twice, which keeps the fused kernel inside the instruction cache.
+template <bool kToSlice, bool kDivide = false, class RowT = Row>
+__device__ __forceinline__ bool decode_group(Smem& sm, const StreamView& sv, const LaneGeom& lg, uint32_t nblk,
+                                             float4 (&v)[8], const RowT& row, int op, float divisor, float& mx,
+                                             float& mn) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  const uint32_t* img = sm.img + (sv.a & 3u);  // see stage_payload
+  const bool tail = __any_sync(kFull, lg.nv != (uint32_t)kSliceVals);
+
+  // offsets of the 32 records: lane b looks at block b
+  bool bad = false;
+  const uint32_t map = sv.map;
+  const uint32_t k = (uint32_t)__popc(map);
+  uint32_t sz_l = 0u;
+  if (lane < nblk) {
+    if ((map >> lane) & 1u) {
+      uint32_t rank = (uint32_t)__popc(map & ((1u << lane) - 1u));
+      sz_l = (rank < 2u * sv.gw) ? reinterpret_cast<const uint16_t*>(img)[rank] : 0u;
+    } else {
+      sz_l = 4u;
+    }
+  }
+  const uint32_t incl_sz = warp_scan_u32(sz_l, lane);
+  const uint32_t off_l = 2u * k + incl_sz - sz_l;
+  const uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
+  if (((raw + 3u) >> 2) != sv.gw) bad = true;  // the same verdict in every thread
+  const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
+  const uint32_t size_blk = __shfl_sync(kFull, sz_l, lg.blk);
+  const bool nonconst = lg.m_blk != 0u && ((map >> lg.blk) & 1u);
+
+  // header, lead codes and stored-byte count of the lane
+  uint32_t R = 0u, B = 0u, code_lo = 0u, code_hi = 0u, T = 0u, lead_lo = 0u;
+  const uint32_t cbytes = (lg.m_blk + 3u) >> 2;
+  if (!bad && nonconst) {
+    R = img_u8(img, boff + 4u);
+    if (!(R >= 10u && R <= 32u)) bad = true;
+    B = (R + 7u) >> 3;
+    if (8u * lg.t < cbytes) {
+      uint32_t o = boff + 5u + 8u * lg.t;
+      uint32_t w = o >> 2, z = 8u * (o & 3u);
+      uint32_t a0 = img[w], a1 = img[w + 1], a2 = img[w + 2];
+      code_lo = __funnelshift_r(a0, a1, z);
+      code_hi = __funnelshift_r(a1, a2, z);
+      if (tail) {
+        // only cbytes code bytes exist; codes of values past the end must be zero
+        uint32_t vb = cbytes - 8u * lg.t;  // valid code bytes of this lane (>= 1)
+        if (vb < 8u) {
+          if (vb <= 4u) {
+            code_hi = 0u;
+            if (vb < 4u) code_lo &= (1u << (8u * vb)) - 1u;
+          } else {
+            code_hi &= (1u << (8u * (vb - 4u))) - 1u;
+          }
+        }
+        if (lg.nv < (uint32_t)kSliceVals) {
+          uint64_t c = ((uint64_t)code_hi << 32) | code_lo;
+          if (c >> (2u * lg.nv)) bad = true;
+        }
+      }
+    }
+    if (B == 2u && ((code_lo & (code_lo >> 1) & 0x55555555u) | (code_hi & (code_hi >> 1) & 0x55555555u)))
+      bad = true;  // lead 3 cannot occur in a 2-byte field
+    lead_lo = sum_fields(code_lo);
+    T = B * lg.nv - lead_lo - sum_fields(code_hi);
+    if (bad) T = 0u;
+  }
+  uint32_t total;
+  const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
+  if (nonconst && !bad && size_blk != 5u + cbytes + total) bad = true;
+  TL(12);
+  if (__syncthreads_or(bad ? 1 : 0)) return false;
+  TL(13);
+
+  // Summary of the lane's values for the predecessor chain: for each byte of the code field, the byte the
+  // LAST value of the lane that stores it holds (found from the lead codes alone, then fetched).
+  const uint32_t pos0 = boff + 5u + cbytes + excl;  // image offset of the lane's first stored byte
+  uint32_t sval = 0u, smask = 0u;
+  if (nonconst && lg.nv != 0u) {
+    SummaryIn si;
+    si.lo = code_lo;
+    si.hi = code_hi;
+    si.lo1 = code_lo >> 1;
+    si.hi1 = code_hi >> 1;
+    si.vlo = 0x55555555u;  // one marker bit per valid value
+    si.vhi = 0x55555555u;
+    if (tail) {
+      si.vlo = lg.nv < 16u ? ((1u << (2u * lg.nv)) - 1u) & 0x55555555u : 0x55555555u;
+      si.vhi = lg.nv <= 16u ? 0u : (lg.nv < 32u ? ((1u << (2u * (lg.nv - 16u))) - 1u) & 0x55555555u : 0x55555555u);
+    }
+    si.lead_lo = lead_lo;
+    si.B = B;
+    si.pos0 = pos0;
+    summary_byte<0>(img, si, sval, smask);
+    if (B > 1u) summary_byte<1>(img, si, sval, smask);
+    if (B > 2u) summary_byte<2>(img, si, sval, smask);
+    if (B > 3u) summary_byte<3>(img, si, sval, smask);
+  }
+  // carry the summaries across the quad: what a lane does not store itself comes from its left
+  {
+    uint32_t tv = __shfl_up_sync(kFull, sval, 1), tm = __shfl_up_sync(kFull, smask, 1);
+    if (lg.t >= 1u) {
+      sval |= tv & ~smask;
+      smask |= tm;
+    }
+    tv = __shfl_up_sync(kFull, sval, 2);
+    tm = __shfl_up_sync(kFull, smask, 2);
+    if (lg.t >= 2u) {
+      sval |= tv & ~smask;
+      smask |= tm;
+    }
+  }
+  uint32_t prev = __shfl_up_sync(kFull, sval, 1);
+  if (lg.t == 0u) prev = 0u;
+  TL(14);
+
+  // the lane's 32 values
+  const float mu = (lg.m_blk != 0u) ? __uint_as_float(img_u32(img, boff)) : 0.0f;
+  constexpr int kUnroll = kToSlice ? 2 : 8;
+  auto put = [&](int j, const float4& r) {
+    if (kToSlice) {
+      const float4 a = row.quad(j);
+      const float4 o = make_float4(reduce_op<kDivide>(r.x, a.x, op, divisor), reduce_op<kDivide>(r.y, a.y, op, divisor),
+                                   reduce_op<kDivide>(r.z, a.z, op, divisor), reduce_op<kDivide>(r.w, a.w, op, divisor));
+      row.set_quad(j, o);
+      mx = max3_nan(max3_nan(mx, o.x, o.y), o.z, o.w);  // the encoder's min/max, while the values are at hand
+      mn = min3_nan(min3_nan(mn, o.x, o.y), o.z, o.w);
+    } else {
+      v[j] = r;
+    }
+  };
+  if (!nonconst) {
+#pragma unroll kUnroll
+    for (int j = 0; j < 8; ++j) put(j, make_float4(mu, mu, mu, mu));
+    return true;
+  }
+  const uint64_t codes = ((uint64_t)code_hi << 32) | code_lo;
+  const uint32_t sh = 32u - R;
+  uint32_t pos = pos0;
+  if (!tail && R <= 24u) {
+    // Fast path: complete slice, field of at most 3 bytes.  A value is assembled by ONE byte permutation of
+    // (predecessor, next four stream bytes): it takes the top `lead` bytes of the field from the predecessor
+    // and the stored bytes, most significant first, from the stream.  The permutation depends only on the
+    // number of stored bytes nb (0..3) and is itself picked, by a byte permutation, from a two-register table.
+    const uint32_t c8B = 8u * B;
+    const uint32_t msh = 1u << sh;  // q << sh == q * 2^sh
+    const uint32_t kSel01 = 0x32143210u, kSel23 = 0x34563245u;  // byte selectors for nb = 0, 1 | 2, 3
+    const uint32_t kPick = 0x10u + 0x22u * B;                   // picks table entry nb = B - lead
+    const uint32_t m8 = opaque(0u - 8u);  // a multiplier the compiler cannot see: c = c8B - 8 l stays ONE multiply-add
+#pragma unroll kUnroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
+      const uint32_t l0 = cb & 3u, l1 = (cb >> 2) & 3u, l2 = (cb >> 4) & 3u, l3 = cb >> 6;
+      const uint32_t c0 = mad_lo(l0, m8, c8B), c1 = mad_lo(l1, m8, c8B), c2 = mad_lo(l2, m8, c8B);  // 8 * stored bytes
+      const uint32_t wi = pos >> 2, z = 8u * pos;  // the funnel shifts use z mod 32 = 8 * (pos & 3)
+      const uint32_t A0 = img[wi], A1 = img[wi + 1], A2 = img[wi + 2], A3 = img[wi + 3];
+      // at most 12 bytes per quad here: three words of string are enough
+      const uint32_t S0 = __funnelshift_r(A0, A1, z), S1 = __funnelshift_r(A1, A2, z), S2 = __funnelshift_r(A2, A3, z);
+      pos += 4u * B - (l0 + l1 + l2 + l3);
+      const uint32_t U0 = __funnelshift_r(S0, S1, c0), U1 = __funnelshift_r(S1, S2, c0);
+      const uint32_t X0 = __funnelshift_r(U0, U1, c1);
+      const uint32_t X1 = __funnelshift_r(U1, S2 >> c0, c1);
+      const uint32_t r3 = __funnelshift_r(X0, X1, c2);
+      const uint32_t q0 = prmt(prev, S0, prmt(kSel01, kSel23, kPick - 0x22u * l0));
+      const uint32_t q1 = prmt(q0, U0, prmt(kSel01, kSel23, kPick - 0x22u * l1));
+      const uint32_t q2 = prmt(q1, X0, prmt(kSel01, kSel23, kPick - 0x22u * l2));
+      const uint32_t q3 = prmt(q2, r3, prmt(kSel01, kSel23, kPick - 0x22u * l3));
+      prev = q3;
+      put(j, make_float4(__fadd_rn(__uint_as_float(q0 * msh), mu), __fadd_rn(__uint_as_float(q1 * msh), mu),
+                         __fadd_rn(__uint_as_float(q2 * msh), mu), __fadd_rn(__uint_as_float(q3 * msh), mu)));
+    }
+    return true;
+  }
+  // General path (ragged slice, 4-byte field, lossless block): one out-of-line call per quad.
+  DecodeCursor cur = {pos0, prev};
+#pragma unroll kUnroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t cb = (uint32_t)(codes >> (8 * j)) & 0xffu;
+    const uint32_t done = 4u * (uint32_t)j;
+    put(j, decode_quad_generic(img, cur, cb, R, mu, lg.nv > done ? lg.nv - done : 0u));
+  }
+  return true;
+}
+
+// Ask L2 for the payload of group gp of the stream (a later CTA will stage it).  The two directory words
+// are loaded by the caller early (dir_a, dir_e); nothing is validated here, a prefetch cannot fault.
+__device__ __forceinline__ void prefetch_payload(const StreamView& sv, uint32_t dir_a, uint32_t dir_e) {
+  if (dir_e <= dir_a || dir_e - dir_a > (uint32_t)kMaxGroupBytes / 4u || dir_e > sv.pw) return;
+  const uint8_t* base = reinterpret_cast<const uint8_t*>(sv.words) + sv.base;
+  for (uint32_t off = 4u * dir_a + 128u * threadIdx.x; off < 4u * dir_e; off += 128u * kThreads)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+}
+
+// Stage group payload words [a, a+gw) of the stream into the image.  The copy starts at the 16-byte boundary
+// at or below word a, so payload word j lands at img[(a & 3) + j] — decode_group reads the image through that
+// shifted origin.  Where every 16-byte piece lies inside the stream (all groups but, at most, a stream's
+// last), one thread hands the whole copy to the bulk-copy engine (`cp.async.bulk`, completion on `bar`): no
+// load, no shared-memory store and no register passes through the lanes.  Returns true in that case: after
+// the CTA's next barrier every thread waits with tma_wait_tile(bar).  Otherwise the words are copied by the
+// lanes and the CTA's next barrier completes the staging.
+__device__ __forceinline__ bool stage_payload(uint32_t* img, const StreamView& sv, uint64_t* bar) {
+  const uint32_t shift = sv.a & 3u;
+  const uint32_t start = sv.a - shift;                // aligned first word
+  const uint32_t n_words = sv.gw + shift;             // words to bring in, from the aligned start
+  const uint32_t n4 = (n_words + 3u) >> 2;            // 16-byte pieces
+  const uint32_t* src = sv.words + (sv.base >> 2) + start;
+  if (n4 != 0u && start + 4u * n4 <= sv.pw && (reinterpret_cast<uintptr_t>(src) & 15u) == 0u) {  // uniform
+    if (threadIdx.x == 0) {
+      const uint32_t b = smem_u32(bar), bytes = 16u * n4;
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_proxy_async();
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                       smem_u32(img)),
+                   "l"(src), "r"(bytes), "r"(b)
+                   : "memory");
+    }
+    return true;
+  }
+#pragma unroll 4
+  for (uint32_t w = threadIdx.x; w < n_words; w += kThreads) img[w] = __ldcs(src + w);
+  return false;
+}
+
+}  // namespace
+}  // namespace ccoll

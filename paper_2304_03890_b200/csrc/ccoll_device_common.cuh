@@ -1,0 +1,408 @@
+// ccoll_device_common.cuh — what every kernel of libccoll shares: small PTX helpers, the geometry of jobs,
+// groups and lanes, the shared-memory layout of a CTA, and the group's values as rows that either the lanes
+// or the TMA unit move.  Included by ccoll_kernels.cu only (one translation unit; everything here is
+// internal to it).
+#pragma once
+#include "ccoll_kernels.cuh"
+
+#include <cuda.h>  // CUtensorMap (a type only; nothing links libcuda)
+
+namespace ccoll {
+#ifdef CCOLL_TIMELINE  // development aid: per-CTA phase timestamps (never compiled into the shipped library)
+__device__ unsigned long long g_timeline[8192 * 16];
+#define TL(slot)                                                                   \
+  do {                                                                             \
+    if (threadIdx.x == 0 && blockIdx.x < 8192 && blockIdx.y == 0 && blockIdx.z == 0) { \
+      unsigned long long t_;                                                       \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                       \
+      g_timeline[blockIdx.x * 16 + (slot)] = t_;                                    \
+    }                                                                              \
+  } while (0)
+#else
+#define TL(slot) do {} while (0)
+#endif
+namespace {
+constexpr uint32_t kFull = 0xffffffffu;
+constexpr int kSliceVals = 32;                      // values per lane
+constexpr int kRowsBytes = kThreads * kSliceVals * 4;  // 16384: one 128-byte row per lane, no padding (swizzled)
+
+// ---------------------------------------------------------------------------------------------------
+// small helpers
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float max_nan(float a, float b) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ float min_nan(float a, float b) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+// three-input forms (sm_100): fold two new values into a running extreme with one instruction
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float min3_nan(float a, float b, float c) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// Byte permutation with a selector that is known to be well formed (every nibble 0..7): the intrinsic
+// __byte_perm masks a run-time selector first, one more integer instruction per use.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+__device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t opaque(uint32_t v) {  // hides a constant from the optimiser
+  asm("" : "+r"(v));
+  return v;
+}
+__device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t* p) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(uint64_t* p, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+// Programmatic dependent launch.  `grid_release` lets a grid launched behind this one (with the programmatic
+// attribute) start filling SM slots as soon as every CTA of this grid has begun; `grid_acquire` holds such a grid
+// until the grid before it has finished and its writes are visible.  Without the attribute both do nothing.
+__device__ __forceinline__ void grid_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_acquire() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ uint64_t pack_state(uint32_t epoch, uint32_t flag, uint32_t value) {
+  return ((uint64_t)epoch << 32) | ((uint64_t)flag << 30) | (uint64_t)(value & kValueMask);
+}
+__device__ __forceinline__ void raise(uint32_t* status, uint32_t code) { atomicMax(status, code); }
+__device__ __forceinline__ uint32_t payload_base(uint32_t G) { return (kHeaderBytes + 8u * G + 4u + 15u) & ~15u; }
+
+// unaligned reads from a word image in shared memory
+__device__ __forceinline__ uint32_t img_u32(const uint32_t* img, uint32_t byte_off) {
+  uint32_t w = byte_off >> 2;
+  return __funnelshift_r(img[w], img[w + 1], 8u * (byte_off & 3u));
+}
+__device__ __forceinline__ uint32_t img_u8(const uint32_t* img, uint32_t byte_off) {
+  return (img[byte_off >> 2] >> (8u * (byte_off & 3u))) & 0xffu;
+}
+// The outgoing image is zeroed once and its shared words are filled by atomic OR, so bytes of one word
+// may come from any lane.
+__device__ __forceinline__ void or_u8(uint32_t* img, uint32_t off, uint32_t byte) {
+  atomicOr(&img[off >> 2], (byte & 0xffu) << (8u * (off & 3u)));
+}
+__device__ __forceinline__ void or_u32(uint32_t* img, uint32_t off, uint32_t v) {
+  uint32_t z = 8u * (off & 3u), w = off >> 2;
+  atomicOr(&img[w], v << z);
+  if (z) atomicOr(&img[w + 1], v >> (32u - z));
+}
+__device__ __forceinline__ void or_u64(uint32_t* img, uint32_t off, uint32_t lo, uint32_t hi) {
+  uint32_t z = 8u * (off & 3u), w = off >> 2;
+  atomicOr(&img[w], lo << z);
+  atomicOr(&img[w + 1], __funnelshift_l(lo, hi, z));
+  if (z) atomicOr(&img[w + 2], hi >> (32u - z));
+}
+
+// ---------------------------------------------------------------------------------------------------
+// geometry
+// ---------------------------------------------------------------------------------------------------
+struct JobGeom {
+  uint32_t lo;      // first value of the job inside the rank buffer
+  uint32_t len;     // values in the job
+  uint32_t nb;      // blocks
+  uint32_t G;       // groups
+  uint32_t m_last;  // values in the job's last block (1..128; 0 if the job is empty)
+};
+// A rank buffer holds at most 2^29 values (the entry points check it), so value indices fit 32 bits.
+__device__ __forceinline__ JobGeom job_geom(uint64_t n64, uint64_t C64, uint32_t y) {
+  JobGeom j;
+  const uint32_t n = (uint32_t)n64, C = (uint32_t)C64;
+  const uint64_t lo64 = (uint64_t)y * C;
+  j.lo = lo64 < n ? (uint32_t)lo64 : n;
+  j.len = min(C, n - j.lo);
+  j.nb = (j.len + kL - 1) / kL;
+  j.G = (j.nb + kGroupBlocks - 1) / kGroupBlocks;
+  j.m_last = j.len - (j.nb ? j.nb - 1 : 0) * kL;
+  return j;
+}
+// What a thread owns in group g: its block's value count and its own valid values.
+struct LaneGeom {
+  uint32_t blk;    // block inside the group (tid / 4)
+  uint32_t t;      // slice inside the block (tid % 4)
+  uint32_t m_blk;  // values in the block (0 = the block does not exist)
+  uint32_t nv;     // valid values in this lane's slice (0..32)
+};
+__device__ __forceinline__ LaneGeom lane_geom(const JobGeom& jg, uint32_t g) {
+  LaneGeom lg;
+  const uint32_t tid = threadIdx.x;
+  lg.blk = tid >> 2;
+  lg.t = tid & 3u;
+  uint32_t gblk = g * kGroupBlocks + lg.blk;
+  lg.m_blk = gblk < jg.nb ? (gblk == jg.nb - 1 ? jg.m_last : (uint32_t)kL) : 0u;
+  int nv = (int)lg.m_blk - (int)(kSliceVals * lg.t);
+  lg.nv = (uint32_t)(nv < 0 ? 0 : (nv > kSliceVals ? kSliceVals : nv));
+  return lg;
+}
+// values of group g that exist (4096 except in the job's last group)
+__device__ __forceinline__ uint32_t group_count(const JobGeom& jg, uint32_t g) {
+  return min((uint32_t)kGroupValues, jg.len - g * (uint32_t)kGroupValues);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// shared memory
+// ---------------------------------------------------------------------------------------------------
+// Dynamic shared memory of a CTA: this control block, then one or two `rows` buffers of kRowsBytes (one
+// padded 144-byte slice per thread: fp32 in, staged bytes, fp32 out).
+struct Smem {
+  alignas(128) uint32_t img[kImgWords];  // payload image of the incoming / outgoing group
+  uint32_t blk_size[kGroupBlocks];       // record bytes, 0 = absent block
+  uint32_t blk_R[kGroupBlocks];          // 0 = constant or absent block
+  uint32_t prefix;                       // exclusive prefix of this group, in words
+  uint32_t fail;
+  alignas(8) uint64_t bar;               // mbarrier the TMA load of the rows completes on
+  uint64_t bar_in;                       // mbarrier the bulk copy of the incoming payload completes on
+};
+constexpr int kCtlBytes = (sizeof(Smem) + 1023) / 1024 * 1024;  // the rows behind it need 1024-byte alignment
+extern __shared__ __align__(1024) uint8_t dyn_smem[];
+// decode kernel: image (aliased by the output rows) at offset 0, then its mbarrier
+constexpr int kDecodeBarOffset = kRowsBytes > (int)sizeof(uint32_t) * kImgWords ? kRowsBytes : (int)sizeof(uint32_t) * kImgWords;
+
+// The image is built with atomic ORs, so it must start as zeros.  Only its front (10 KB, more than most
+// groups need) is cleared up front; a group whose payload turns out longer clears the rest once its size is
+// known (zero_image_rest), at the price of one more barrier.
+constexpr int kZeroFrontWords = 5 * 4 * kThreads;  // five 128-bit stores per thread
+constexpr int kZeroSlackWords = 8;                 // words past the payload that placement may touch
+__device__ __forceinline__ void zero_image(uint32_t* img) {  // a barrier must follow
+  uint4* p = reinterpret_cast<uint4*>(img) + threadIdx.x;
+#pragma unroll
+  for (int r = 0; r < kZeroFrontWords / (4 * kThreads); ++r) p[r * kThreads] = make_uint4(0u, 0u, 0u, 0u);
+}
+__device__ __forceinline__ void zero_image_rest(uint32_t* img) {  // whole CTA; ends with a barrier
+  for (int v = kZeroFrontWords / 4 + (int)threadIdx.x; v < kImgWords / 4; v += kThreads)
+    reinterpret_cast<uint4*>(img)[v] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+}
+
+// Ask L2 for the fp32 values of a group that a later CTA will load (one 128-byte line per thread).  Issued by
+// the CTA that currently occupies the SM slot that later CTA will get, so its loads find the data in L2.
+__device__ __forceinline__ void prefetch_group(const float* x, const JobGeom& jg, uint32_t g) {
+  if (g >= jg.G) return;
+  const uint32_t first = g * (uint32_t)kGroupValues + 32u * threadIdx.x;
+  if (first < jg.len) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + first));
+}
+
+// ---- rows: the group's values as a tile the TMA unit moves ---------------------------------------------
+// A group of 4096 fp32 values is a tile of 128 rows x 128 bytes, row t = the 32 values of lane t.  The TMA unit
+// moves such a tile between global and shared memory in one instruction, past the load/store pipe, and applies
+// the 128-byte swizzle on the way: inside every 1024-byte span the 16-byte piece j of row r sits at piece
+// j ^ (r & 7).  A lane that walks its own row piece by piece then meets no bank conflict although the rows
+// are only 128 bytes apart (no padding).  Byte offset o < 128 of row t is at  128 t + (o ^ 16 (t & 7))  =
+// (128 t + 16 (t & 7)) ^ o : one XOR per access.
+struct Row {
+  uint8_t* tile;  // the rows buffer (1024-byte aligned)
+  uint32_t off;   // 128 t + 16 (t & 7)
+  __device__ __forceinline__ float4 quad(uint32_t j) const {
+    return *reinterpret_cast<const float4*>(tile + (off ^ (16u * j)));
+  }
+  __device__ __forceinline__ void set_quad(uint32_t j, const float4& v) const {
+    *reinterpret_cast<float4*>(tile + (off ^ (16u * j))) = v;
+  }
+};
+__device__ __forceinline__ Row row_of(uint8_t* rows, uint32_t t) { return Row{rows, 128u * t + 16u * (t & 7u)}; }
+// The other way to keep a lane's walk over its row free of bank conflicts: rows 144 bytes apart, no swizzle, no
+// XOR per access.  The TMA unit makes this layout too: a box 36 values wide over a tensor whose rows have 32
+// lands as rows of 144 bytes (the four values past the row's end are out of bounds and arrive as zeros; a
+// store does not write them).  The encoder and the fused round use it (their integer pipe is the busy one,
+// and the spare words of a row let lanes stagger their staged output); the decoder's output tile is swizzled
+// (16 KB instead of 18 KB: that is what lets 12 of its CTAs share an SM).  Same interface as Row.
+constexpr int kPaddedRowBytes = 144;
+constexpr int kPaddedRowsBytes = kThreads * kPaddedRowBytes;  // 18432
+struct PaddedRow {
+  static constexpr uint32_t kWords = 36u;
+  // Staged words start `rot` words into the row: with rows 36 words apart, lanes l and l + 8 would otherwise
+  // hit the same bank whenever they are at the same word; lane l's word w now sits in bank 4 l + l/8 + w.
+  __device__ static __forceinline__ uint32_t rot(uint32_t t) { return (t >> 3) & 3u; }
+  uint8_t* p;
+  __device__ __forceinline__ float4 quad(uint32_t j) const { return *reinterpret_cast<const float4*>(p + 16u * j); }
+  __device__ __forceinline__ void set_quad(uint32_t j, const float4& v) const { *reinterpret_cast<float4*>(p + 16u * j) = v; }
+  __device__ __forceinline__ uint4 words4(uint32_t j) const { return *reinterpret_cast<const uint4*>(p + 16u * j); }
+  __device__ __forceinline__ uint32_t word(uint32_t i) const { return *reinterpret_cast<const uint32_t*>(p + 4u * i); }
+  __device__ __forceinline__ void set_word(uint32_t i, uint32_t v) const { *reinterpret_cast<uint32_t*>(p + 4u * i) = v; }
+  __device__ __forceinline__ uint32_t* word_ptr(uint32_t i) const { return reinterpret_cast<uint32_t*>(p + 4u * i); }
+};
+template <class RowT>
+__device__ __forceinline__ RowT make_row(uint8_t* rows, uint32_t t);
+template <>
+__device__ __forceinline__ PaddedRow make_row<PaddedRow>(uint8_t* rows, uint32_t t) {
+  return PaddedRow{rows + kPaddedRowBytes * t};
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// generic-proxy writes to shared memory must be fenced before the TMA unit (async proxy) reads them
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One thread: arm the barrier and ask the TMA unit for rows [row0, row0+128) of plane `plane` of the tensor.
+__device__ __forceinline__ void tma_load_tile(const CUtensorMap* map, uint8_t* rows, uint64_t* bar, uint32_t row0,
+                                              uint32_t plane, uint32_t tile_bytes) {
+  const uint32_t b = smem_u32(bar);
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  fence_proxy_async();
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(tile_bytes) : "memory");
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          smem_u32(rows)),
+      "l"(map), "r"(0), "r"(row0), "r"(plane), "r"(b)
+      : "memory");
+}
+// Every thread that will read the rows: wait for the tile (phase 0 of the barrier).  The wait is bounded;
+// false = it gave up (the caller raises a time-out and does not touch the rows).
+__device__ __forceinline__ bool tma_wait_tile(uint64_t* bar) {
+  const uint32_t b = smem_u32(bar);
+#pragma unroll 1
+  for (uint32_t tries = 0; tries < (1u << 16); ++tries) {
+    uint32_t done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done)
+        : "r"(b)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+// One thread: store the tile to rows [row0, row0+128) of plane `plane` of the tensor; the same thread then
+// calls tma_store_wait() before shared memory is reused or the CTA exits (the tile has been read by then).
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, const uint8_t* rows, uint32_t row0, uint32_t plane) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(0),
+               "r"(row0), "r"(plane), "r"(smem_u32(rows))
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+// Padded rows: every warp reads 512 contiguous bytes per instruction (128-bit streaming loads) and scatters
+// them; in round r thread tid moves the float4 number r*128 + tid of the group, piece (tid & 7) of row
+// 16 r + tid / 8.  Zeros past the end of the data.  A __syncthreads must follow before the rows are read.
+__device__ __forceinline__ void load_rows_padded(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint32_t cnt = group_count(jg, g);
+  const float* src = x + (size_t)g * kGroupValues;
+  float4* dst = reinterpret_cast<float4*>(rows + (tid >> 3) * kPaddedRowBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kPaddedRowBytes / 16;  // float4s between a thread's rounds
+  if (cnt == (uint32_t)kGroupValues) {  // a complete group: no bounds to watch
+    float4 t[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t[r] = __ldcs(reinterpret_cast<const float4*>(src) + r * kThreads + tid);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) dst[r * kRoundStride] = t[r];
+    return;
+  }
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (4u * f + 4u <= cnt) {
+      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
+    } else {
+      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
+    }
+    dst[r * kRoundStride] = v;
+  }
+}
+// The same with every warp loading its own 32 rows (4 KB of the group): in round r lane l moves the float4
+// number 256 w + 32 r + l, piece (l & 7) of row 32 w + 4 r + l / 8.  A warp then depends on its own loads only:
+// a __syncwarp is enough before its lanes read their rows.
+__device__ __forceinline__ void load_rows_padded_own(uint8_t* rows, const float* x, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t cnt = group_count(jg, g);
+  const float* src = x + (size_t)g * kGroupValues;
+  const uint32_t f0 = 256u * warp + lane;  // the thread's float4 of round 0
+  float4* dst = reinterpret_cast<float4*>(rows + (32u * warp + (lane >> 3)) * kPaddedRowBytes + 16u * (lane & 7u));
+  constexpr int kRoundStride = 4 * kPaddedRowBytes / 16;  // float4s between a thread's rounds (four rows)
+  if (cnt == (uint32_t)kGroupValues) {
+    float4 t[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t[r] = __ldcs(reinterpret_cast<const float4*>(src) + f0 + 32 * r);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) dst[r * kRoundStride] = t[r];
+    return;
+  }
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = f0 + 32u * (uint32_t)r;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (4u * f + 4u <= cnt) {
+      v = __ldcs(reinterpret_cast<const float4*>(src) + f);
+    } else {
+      if (4u * f + 0u < cnt) v.x = __ldcs(src + 4u * f + 0u);
+      if (4u * f + 1u < cnt) v.y = __ldcs(src + 4u * f + 1u);
+      if (4u * f + 2u < cnt) v.z = __ldcs(src + 4u * f + 2u);
+    }
+    dst[r * kRoundStride] = v;
+  }
+}
+// A swizzled tile without the TMA unit (a group that is not complete, or no tensor map): coalesced 128-bit
+// streaming stores, bounds watched; thread tid moves the float4 number r*128 + tid in round r, which is piece
+// (tid & 7) of row 16 r + tid / 8.  A __syncthreads must separate it from the writes of the rows.
+__device__ __forceinline__ void store_rows(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint32_t cnt = group_count(jg, g);
+  float* dst = out + (size_t)g * kGroupValues;
+  const uint8_t* src = rows + 128u * (tid >> 3) + 16u * ((tid & 7u) ^ ((tid >> 3) & 7u));
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    const float4 t = *reinterpret_cast<const float4*>(src + 2048 * r);
+    if (4u * f + 4u <= cnt) {
+      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+    } else {
+      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
+      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
+      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+    }
+  }
+}
+// The same from padded rows (fused round: the owner's sums of a group that is not complete).
+__device__ __forceinline__ void store_rows_padded(const uint8_t* rows, float* out, const JobGeom& jg, uint32_t g) {
+  const uint32_t tid = threadIdx.x;
+  const uint32_t cnt = group_count(jg, g);
+  float* dst = out + (size_t)g * kGroupValues;
+  const float4* src = reinterpret_cast<const float4*>(rows + (tid >> 3) * kPaddedRowBytes + 16u * (tid & 7u));
+  constexpr int kRoundStride = (kThreads / 8) * kPaddedRowBytes / 16;
+#pragma unroll 1
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t f = (uint32_t)r * kThreads + tid;
+    const float4 t = src[r * kRoundStride];
+    if (4u * f + 4u <= cnt) {
+      __stcs(reinterpret_cast<float4*>(dst) + f, t);
+    } else {
+      if (4u * f + 0u < cnt) dst[4u * f + 0u] = t.x;
+      if (4u * f + 1u < cnt) dst[4u * f + 1u] = t.y;
+      if (4u * f + 2u < cnt) dst[4u * f + 2u] = t.z;
+    }
+  }
+}
+// Ragged rows: values past the end of the data are replaced by the block's first value, so that they
+// cannot change min or max.  (The first value of block b is the first value of row 4b.)  Whole warp.
+template <class RowT>
+__device__ __forceinline__ void pad_ragged(uint8_t* rows, const LaneGeom& lg) {
+  __syncwarp();
+  if (lg.nv < (uint32_t)kSliceVals) {
+    const uint32_t f = make_row<RowT>(rows, threadIdx.x & ~3u).word(0);
+    const RowT row = make_row<RowT>(rows, threadIdx.x);
+    for (uint32_t i = lg.nv; i < (uint32_t)kSliceVals; ++i) row.set_word(i, f);
+  }
+  __syncwarp();
+}
+
+}  // namespace
+}  // namespace ccoll

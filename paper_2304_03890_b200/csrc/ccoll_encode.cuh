@@ -1,0 +1,417 @@
+// ccoll_encode.cuh — the encoder of a group: block rules, the lane's byte string, placement in the payload
+// image, the exchange of group sizes and the copy-out.  Used by the compress kernel and by the second half of
+// the fused round.  Included by ccoll_kernels.cu only, after ccoll_device_common.cuh.
+#pragma once
+#include "ccoll_device_common.cuh"
+
+namespace ccoll {
+namespace {
+
+// ---------------------------------------------------------------------------------------------------
+// encode side
+// ---------------------------------------------------------------------------------------------------
+// Rules R1-R6 for the lane's block (the four lanes of a block compute the same plan).
+struct Plan {
+  uint32_t R;        // kept bits; 0 = constant (or absent) block, 32 = lossless
+  uint32_t mu_bits;  // representative value
+  float mu;
+  uint32_t sh;       // 32 - R (0 when R is 0 or 32)
+  uint32_t B;        // bytes per code
+  bool lossless;
+};
+
+// Largest and smallest of the lane's 32 values (a NaN wins both), read from the lane's slice.  The loop is
+// unrolled only twice: fully unrolled on register arrays the fused kernel outgrew the 32 KB instruction cache.
+template <class RowT>
+__device__ __forceinline__ void lane_minmax(const RowT& row, float& mx, float& mn) {
+  float4 q = row.quad(0);
+  mx = max3_nan(max_nan(q.x, q.y), q.z, q.w);
+  mn = min3_nan(min_nan(q.x, q.y), q.z, q.w);
+#pragma unroll 2
+  for (int j = 1; j < 8; ++j) {
+    q = row.quad(j);
+    mx = max3_nan(max3_nan(mx, q.x, q.y), q.z, q.w);
+    mn = min3_nan(min3_nan(mn, q.x, q.y), q.z, q.w);
+  }
+}
+__device__ __forceinline__ Plan plan_block(float mx, float mn, const LaneGeom& lg, float eb, int eb_exp) {
+  mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 1));
+  mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 1));
+  mx = max_nan(mx, __shfl_xor_sync(kFull, mx, 2));
+  mn = min_nan(mn, __shfl_xor_sync(kFull, mn, 2));
+  const float kInf = __uint_as_float(0x7f800000u);
+  bool special = !(fabsf(mx) < kInf) || !(fabsf(mn) < kInf);  // NaN or Inf somewhere in the block
+  float mu = __fadd_rn(__fmul_rn(0.5f, mn), __fmul_rn(0.5f, mx));
+  uint32_t mub = __float_as_uint(mu);
+  if ((mub << 1) == 0u) mub = 0u;  // a zero of either sign becomes +0
+  mu = __uint_as_float(mub);
+  float r = fmaxf(__fsub_rn(mx, mu), __fsub_rn(mu, mn));
+  Plan p;
+  if (lg.m_blk == 0u || (!special && r <= eb)) {
+    p.R = 0u;
+    p.mu_bits = mub;
+    p.mu = mu;
+    p.sh = 0u;
+    p.B = 0u;
+    p.lossless = false;
+    return p;
+  }
+  int m_bits = (int)((__float_as_uint(r) >> 23) & 0xffu) - eb_exp + 1;
+  p.lossless = special || m_bits >= 23;
+  p.R = p.lossless ? 32u : (uint32_t)(9 + m_bits);
+  p.mu_bits = p.lossless ? 0u : mub;
+  p.mu = __uint_as_float(p.mu_bits);
+  p.sh = 32u - p.R;
+  p.B = (p.R + 7u) >> 3;
+  return p;
+}
+
+__device__ __forceinline__ uint32_t code_of(float x, const Plan& p) {
+  return __float_as_uint(p.lossless ? x : __fsub_rn(x, p.mu)) >> p.sh;
+}
+
+// Rules R7-R8 for the lane's 32 values.  The lane's byte string is built in a 64-bit big-endian accumulator
+// (hi:lo; Tb = bits appended so far, the low Tb & 31 of them still waiting): a value's stored bytes are its low
+// n = 8 * (stored bytes) bits, appended with two funnel shifts; whenever 32 bits are complete they leave as
+// one word (byte-reversed, since the first byte of the stream is the most significant one).  n comes
+// straight from the leading-zero count of (code xor predecessor); `fix` forces at least one stored byte when
+// the field is 4 bytes wide (lead is capped at 3).  Values are read from the lane's row quad by quad and the
+// staged words overwrite the row in place, which is safe because at most 16 bytes are staged per quad and
+// quad j is read before anything is written at or behind its position.
+// kGeneral = false: all 32 values valid, block not lossless (loop unrolled twice).  kGeneral = true: ragged
+// rows (values past nv store nothing and have lead code 0) and lossless blocks, rolled.
+template <bool kGeneral, class RowT>
+__device__ __forceinline__ void emit_lane(const RowT& row, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
+                                          uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  const bool lossless = kGeneral && R == 32u;
+  const uint32_t B = (R + 7u) >> 3, sh = 32u - R;
+  const uint32_t fix = (B == 4u) ? 1u : 0u;
+  const uint32_t unused = 4u - B;  // top bytes of the 32-bit code that the field does not have
+  const float mu = __uint_as_float(mu_bits);
+  uint32_t lo = 0u, hi = 0u, Tb = 0u;
+  uint32_t clo = 0u, chi = 0u;
+  const uint32_t rot = RowT::rot(threadIdx.x);  // staged word k goes to word rot + k of the row
+  uint32_t* wp = row.word_ptr(rot);             // where the next completed word goes
+  auto put = [&](uint32_t q, uint32_t sa) {
+    const uint32_t n = 32u - sa;
+    const uint32_t t = __funnelshift_lc(0u, q, sa);  // the stored bits, at the top of the word
+    const uint32_t Tn = Tb + n;                      // the only loop-carried add: everything else hangs off it
+    hi = __funnelshift_lc(lo, hi, n);
+    lo = __funnelshift_lc(t, lo, n);
+    if ((Tn ^ Tb) & 32u)  // a word boundary was crossed (n <= 32: at most one)
+      *wp++ = __byte_perm(__funnelshift_r(lo, hi, Tn), 0u, 0x0123);
+    Tb = Tn;
+  };
+  // the next quad is always read before the current one's words are stored: they may reach rot <= 3 words
+  // into it
+  float4 xn = row.quad(0);
+#pragma unroll(kGeneral ? 1 : 2)
+  for (int j = 0; j < 8; ++j) {
+    const float4 x = xn;
+    xn = row.quad(j < 7 ? j + 1 : 7);
+    const uint32_t q0 = __float_as_uint(lossless ? x.x : __fsub_rn(x.x, mu)) >> sh,
+                   q1 = __float_as_uint(lossless ? x.y : __fsub_rn(x.y, mu)) >> sh,
+                   q2 = __float_as_uint(lossless ? x.z : __fsub_rn(x.z, mu)) >> sh,
+                   q3 = __float_as_uint(lossless ? x.w : __fsub_rn(x.w, mu)) >> sh;
+    uint32_t sa0 = (uint32_t)__clz((q0 ^ prev) | fix) & 0x38u, sa1 = (uint32_t)__clz((q1 ^ q0) | fix) & 0x38u,
+             sa2 = (uint32_t)__clz((q2 ^ q1) | fix) & 0x38u, sa3 = (uint32_t)__clz((q3 ^ q2) | fix) & 0x38u;
+    prev = q3;
+    // lead code of a value = leading zero bytes of the xor, less the unused top bytes of the field; the
+    // quad's four codes enter the 64-bit code string from the top, so that after eight quads quad 0 is lowest
+    uint32_t cb;
+    if (kGeneral) {
+      uint32_t l0 = (sa0 >> 3) - unused, l1 = (sa1 >> 3) - unused, l2 = (sa2 >> 3) - unused, l3 = (sa3 >> 3) - unused;
+      if (4u * j + 0u >= nv) sa0 = 32u, l0 = 0u;
+      if (4u * j + 1u >= nv) sa1 = 32u, l1 = 0u;
+      if (4u * j + 2u >= nv) sa2 = 32u, l2 = 0u;
+      if (4u * j + 3u >= nv) sa3 = 32u, l3 = 0u;
+      cb = (l0 | (l1 << 2) | (l2 << 4) | (l3 << 6)) << 24;
+    } else {
+      cb = ((sa0 + 4u * sa1 + 16u * sa2 + 64u * sa3) << 21) - unused * (85u << 24);
+    }
+    clo = __funnelshift_r(clo, chi, 8u);
+    chi = (chi >> 8) | cb;
+    put(q0, sa0);
+    put(q1, sa1);
+    put(q2, sa2);
+    put(q3, sa3);
+  }
+  const uint32_t pend = Tb & 31u, w = Tb >> 5;
+  // the last partial word, zero padded, and a zero word behind it for the realigning copy — as far as the row
+  // reaches (a row that is full to its last byte has neither; copy_staged reads zeros past the row's end)
+  if (rot + w < RowT::kWords) row.set_word(rot + w, pend ? __byte_perm(lo << (32u - pend), 0u, 0x0123) : 0u);
+  if (rot + w + 1u < RowT::kWords) row.set_word(rot + w + 1u, 0u);
+  T_out = Tb >> 3;
+  code_lo = clo;
+  code_hi = chi;
+}
+template <class RowT>
+__device__ __noinline__ void emit_lane_general(RowT row, uint32_t R, uint32_t mu_bits, uint32_t nv, uint32_t prev,
+                                               uint32_t& T_out, uint32_t& code_lo, uint32_t& code_hi) {
+  emit_lane<true, RowT>(row, R, mu_bits, nv, prev, T_out, code_lo, code_hi);
+}
+
+// Copy the lane's T staged bytes (they start at word rot of its row) to byte offset dst of the image.  The
+// first and last image word may be shared with a neighbour and are ORed in; the words between are plain
+// stores.  The row is read in aligned 128-bit pieces from its start, as a string whose first rot words are
+// to be skipped: row word g goes to image word (dst / 4) - rot + g.
+template <class RowT>
+__device__ __forceinline__ void copy_staged(uint32_t* img, const RowT& row, uint32_t dst, uint32_t T) {
+  if (T == 0u) return;
+  const uint32_t rot = RowT::rot(threadIdx.x);
+  const uint32_t z = 8u * (dst & 3u);
+  uint32_t* out = img + (dst >> 2);                // image word of staged word 0
+  const uint32_t nw = ((dst & 3u) + T + 3u) >> 2;  // image words touched, <= 33
+  atomicOr(&out[0], row.word(rot) << z);
+  if (nw > 1u) {
+    const uint32_t k = rot + nw - 1u;  // nothing is staged past the row's last word
+    const uint32_t last = k < RowT::kWords ? row.word(k) : 0u;
+    atomicOr(&out[nw - 1u], __funnelshift_l(row.word(k - 1u), last, z));
+  }
+  if (nw <= 2u) return;
+  const uint32_t ni = nw - 2u;  // interior image words 1 .. nw-2 = row words rot+1 .. rot+nw-2
+  uint32_t* outr = out - rot;   // image word of row word 0 (never dereferenced below row word rot + 1)
+  uint32_t prevw = 0u;
+  for (uint32_t c = 0; 4u * c <= rot + ni; ++c) {
+    const uint4 cur = row.words4(c);
+    const uint32_t w0 = __funnelshift_l(prevw, cur.x, z), w1 = __funnelshift_l(cur.x, cur.y, z),
+                   w2 = __funnelshift_l(cur.y, cur.z, z), w3 = __funnelshift_l(cur.z, cur.w, z);
+    prevw = cur.w;
+    const uint32_t g = 4u * c - rot;  // staged word index of cur.x (wraps below zero for skipped words)
+    if (g - 1u < ni) outr[4u * c] = w0;
+    if (g < ni) outr[4u * c + 1u] = w1;
+    if (g + 1u < ni) outr[4u * c + 2u] = w2;
+    if (g + 2u < ni) outr[4u * c + 3u] = w3;
+  }
+}
+
+// inclusive warp scan
+__device__ __forceinline__ uint32_t warp_scan_u32(uint32_t v, uint32_t lane) {
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    uint32_t t = __shfl_up_sync(kFull, v, d);
+    if (lane >= (uint32_t)d) v += t;
+  }
+  return v;
+}
+// inclusive scan over the four lanes of a block; total = sum over the quad
+__device__ __forceinline__ uint32_t quad_scan(uint32_t v, uint32_t t, uint32_t lane, uint32_t& total) {
+  uint32_t a = __shfl_up_sync(kFull, v, 1);
+  if (t >= 1u) v += a;
+  a = __shfl_up_sync(kFull, v, 2);
+  if (t >= 2u) v += a;
+  total = __shfl_sync(kFull, v, lane | 3u);
+  return v;
+}
+
+// Place of a group in its stream = sum of the sizes of all groups before it.  A chained look-back (wait
+// for the predecessor's inclusive prefix) advances at most one window of tiles per L2 round trip, which
+// caps a kernel of 8192 tiles at ~100 us whatever its work.  Instead sizes are summed on two levels and
+// nothing ever waits on a prefix: A[t] = size of tile t; SA[s] = size of super-tile s (32 tiles), written
+// by the super-tile's last tile from the A's it has to read anyway.  Tile g needs A[32s .. g-1] and
+// SA[0 .. s-1]: independent loads spread over the CTA's threads, one round trip once the data is there.
+// (A third level, sums of 1024 tiles, cuts the loads per tile from G/64 to about 36 and was measured slower.)
+// Words carry the launch's epoch, so stale entries read as "not written yet"; every wait is bounded.
+__device__ __forceinline__ uint32_t poll_size(const uint64_t* p, uint32_t epoch, uint32_t* status, bool& bad) {
+  uint32_t spins = 0;
+  while (true) {
+    const uint64_t w = ld_relaxed_u64(p);
+    if ((uint32_t)(w >> 32) == epoch) {
+      if (((uint32_t)(w >> 30) & 3u) == kFlagPoison) bad = true;
+      return (uint32_t)w & kValueMask;
+    }
+    if (++spins > kSpinLimit) {
+      raise(status, kErrTimeout);
+      bad = true;
+      return 0u;
+    }
+    __nanosleep(32);
+  }
+}
+// Both halves add to sm.prefix and raise sm.fail on a poisoned or timed-out entry; both words are read after
+// the next barrier.  Called by every thread of the CTA after A[g] was published.
+// Warp 0: the sizes of the earlier tiles of the own super-tile; the super-tile's last tile also publishes
+// SA[s].  That tile calls this BEFORE it places its bytes in the image, every other tile after: the tiles of
+// the next super-tile then find SA[s] one round trip after A[32s+31] instead of one placement and a round
+// trip later.
+struct SizeWords {
+  uint64_t *A, *SA;
+};
+__device__ __forceinline__ SizeWords size_words(const EncodeBatch& b, uint32_t y) {
+  SizeWords w;
+  w.A = b.tile_state + (uint64_t)y * b.state_stride;
+  w.SA = w.A + b.tiles_per_job;
+  return w;
+}
+__device__ __forceinline__ void prefix_own_super_tile(Smem& sm, const SizeWords& w, uint32_t g, uint32_t G,
+                                                      uint32_t words, uint32_t epoch, uint32_t* status) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  if (tid >= 32u) return;
+  const uint32_t s = g >> 5, r = g & 31u;
+  uint32_t sum = 0u;
+  bool bad = false;
+  if (lane < r) sum = poll_size(&w.A[32u * s + lane], epoch, status, bad);
+  sum = __reduce_add_sync(kFull, sum);
+  bad = __any_sync(kFull, bad);
+  if (lane == 0) {
+    if (r == 31u || g == G - 1u)
+      st_relaxed_u64(&w.SA[s], pack_state(epoch, bad ? kFlagPoison : kFlagAggregate, sum + words));
+    if (sum) atomicAdd(&sm.prefix, sum);
+    if (bad) atomicOr(&sm.fail, 1u);
+  }
+}
+// Warps 1-3: the earlier super-tiles.
+__device__ __forceinline__ void prefix_earlier_super_tiles(Smem& sm, const SizeWords& w, uint32_t g, uint32_t epoch,
+                                                           uint32_t* status) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  if (tid < 32u) return;
+  const uint32_t s = g >> 5;
+  uint32_t sum = 0u;
+  bool bad = false;
+  for (uint32_t t = tid - 32u; t < s; t += kThreads - 32u) sum += poll_size(&w.SA[t], epoch, status, bad);
+  sum = __reduce_add_sync(kFull, sum);
+  bad = __any_sync(kFull, bad);
+  if (lane == 0) {
+    if (sum) atomicAdd(&sm.prefix, sum);
+    if (bad) atomicOr(&sm.fail, 1u);
+  }
+}
+
+// Encode the group whose values wait in the lanes' slices (ragged slices already padded; mx, mn = largest and
+// smallest value of the lane's slice): build the payload image, find its place in the stream and copy it
+// out.  The image must have been zeroed (that is made visible by the barrier inside) before the call.
+template <class RowT>
+__device__ __forceinline__ void encode_group(Smem& sm, uint8_t* rows, const LaneGeom& lg, const EncodeBatch& b,
+                                             const JobGeom& jg, uint32_t g, uint32_t y, uint8_t* sout, float mx,
+                                             float mn, bool tail) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const RowT row = make_row<RowT>(rows, tid);
+  Plan p = plan_block(mx, mn, lg, b.eb, b.eb_exp);
+  // code of the value just before this lane's first one (0 at the start of a block)
+  uint32_t prev = __shfl_up_sync(kFull, code_of(__uint_as_float(row.word(kSliceVals - 1)), p), 1);
+  if (lg.t == 0u) prev = 0u;
+  uint32_t T = 0u, code_lo = 0u, code_hi = 0u;
+  if (p.R != 0u) {
+    if (tail || p.lossless)
+      emit_lane_general(row, p.R, p.mu_bits, lg.nv, prev, T, code_lo, code_hi);
+    else
+      emit_lane<false, RowT>(row, p.R, p.mu_bits, (uint32_t)kSliceVals, prev, T, code_lo, code_hi);
+  }
+  uint32_t total;
+  const uint32_t excl = quad_scan(T, lg.t, lane, total) - T;
+  const uint32_t cbytes = (lg.m_blk + 3u) >> 2;  // lead-code bytes of the block
+  if (lg.t == 0u) {
+    sm.blk_size[lg.blk] = lg.m_blk == 0u ? 0u : (p.R ? 5u + cbytes + total : 4u);
+    sm.blk_R[lg.blk] = p.R;
+  }
+  __syncthreads();  // sizes visible; also: image zero-fill and all staging done
+  TL(4);
+
+  // every warp derives the offsets of all 32 records (cheap, and saves a barrier)
+  const uint32_t sz_l = sm.blk_size[lane];
+  const uint32_t R_l = sm.blk_R[lane];
+  const uint32_t bitmap = __ballot_sync(kFull, R_l != 0u);
+  const uint32_t k = (uint32_t)__popc(bitmap);
+  const uint32_t incl_sz = warp_scan_u32(sz_l, lane);
+  const uint32_t off_l = 2u * k + incl_sz - sz_l;
+  const uint32_t raw = 2u * k + __shfl_sync(kFull, incl_sz, 31);
+  const uint32_t words = (raw + 3u) >> 2;
+  const uint32_t boff = __shfl_sync(kFull, off_l, lg.blk);
+  if (words + (uint32_t)kZeroSlackWords > (uint32_t)kZeroFrontWords) zero_image_rest(sm.img);  // rare, uniform
+
+  const SizeWords sw = size_words(b, y);
+  if (warp == 0) {
+    if (lane == 0) st_relaxed_u64(&sw.A[g], pack_state(b.epoch, kFlagAggregate, words));
+    if (R_l != 0u) {
+      uint32_t rank = (uint32_t)__popc(bitmap & ((1u << lane) - 1u));
+      atomicOr(&sm.img[rank >> 1], sz_l << (16u * (rank & 1u)));
+    }
+  }
+  const bool closes = (g & 31u) == 31u || g == jg.G - 1u;  // this tile completes its super-tile
+  if (closes) prefix_own_super_tile(sm, sw, g, jg.G, words, b.epoch, b.status);
+  if (lg.m_blk != 0u) {
+    if (lg.t == 0u) {
+      or_u32(sm.img, boff, p.mu_bits);
+      if (p.R) or_u8(sm.img, boff + 4u, p.R);
+    }
+    if (p.R) {
+      if (8u * lg.t < cbytes) or_u64(sm.img, boff + 5u + 8u * lg.t, code_lo, code_hi);
+      copy_staged(sm.img, row, boff + 5u + cbytes + excl, T);
+    }
+  }
+
+  // place of the group in the stream
+  TL(5);
+  if (!closes) prefix_own_super_tile(sm, sw, g, jg.G, words, b.epoch, b.status);
+  prefix_earlier_super_tiles(sm, sw, g, b.epoch, b.status);
+  TL(11);
+  __syncthreads();
+  TL(6);
+  const uint32_t prefix = sm.prefix;
+  if (sm.fail) return;
+  const uint32_t base = payload_base(jg.G);
+  const uint64_t end = (uint64_t)base + 4ull * ((uint64_t)prefix + words);
+  uint32_t* out32 = reinterpret_cast<uint32_t*>(sout);
+  if (end > b.out_cap) {
+    if (tid == 0) raise(b.status, kErrCapacity);
+    return;
+  }
+  {
+    // coalesced copy-out: consecutive lanes move consecutive words (conflict-free shared reads, full
+    // 128-byte lines per warp store)
+    uint32_t* dst = out32 + (base >> 2) + prefix;
+    TL(8);
+    for (uint32_t j = tid; j < words; j += kThreads) __stcs(dst + j, sm.img[j]);
+    TL(9);
+  }
+  if (tid == 0) {
+    out32[8 + g] = prefix;             // dir[g]
+    out32[8 + jg.G + 1 + g] = bitmap;  // bitmap[g]
+  }
+  TL(10);
+  if (g == 0 && tid >= 32 && tid < 32 + 4) {
+    // static part of the header and the zero pad between the bitmap and the payload
+    uint32_t t = tid - 32;
+    if (t == 0) {
+      out32[0] = kMagic;
+      out32[1] = 0u;
+      out32[2] = jg.len;
+      out32[3] = 0u;
+      out32[4] = (uint32_t)kL;
+      out32[5] = __float_as_uint(b.eb);
+    }
+    for (uint32_t w = 8 + 2 * jg.G + 1 + t; w < (base >> 2); w += 4) out32[w] = 0u;
+  }
+  if (g == jg.G - 1 && tid == 64) {
+    out32[8 + jg.G] = prefix + words;  // dir[G]
+    out32[6] = (uint32_t)end;
+    out32[7] = (uint32_t)(end >> 32);
+    if (b.out_bytes) b.out_bytes[y] = end;
+    if (b.moved) atomicAdd(reinterpret_cast<unsigned long long*>(b.moved), (unsigned long long)b.moved_mult * end);
+  }
+}
+
+// An empty job still yields a valid 48-byte stream.
+__device__ __forceinline__ void write_empty_stream(const EncodeBatch& b, uint32_t y, uint8_t* sout) {
+  if (threadIdx.x != 0) return;
+  if (b.out_cap < 48u) {
+    raise(b.status, kErrCapacity);
+    return;
+  }
+  uint32_t* out32 = reinterpret_cast<uint32_t*>(sout);
+  out32[0] = kMagic;
+  out32[1] = 0u;
+  out32[2] = 0u;
+  out32[3] = 0u;
+  out32[4] = (uint32_t)kL;
+  out32[5] = __float_as_uint(b.eb);
+  out32[6] = 48u;
+  out32[7] = 0u;
+  out32[8] = 0u;  // dir[0]
+  out32[9] = out32[10] = out32[11] = 0u;
+  if (b.out_bytes) b.out_bytes[y] = 48u;
+  if (b.moved) atomicAdd(reinterpret_cast<unsigned long long*>(b.moved), (unsigned long long)b.moved_mult * 48ull);
+}
+
+}  // namespace
+}  // namespace ccoll
