@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(kThreads, 6) ccoll_compress_kernel(const __gri
   if (tail) pad_ragged<PaddedRow>(rows, lg);
   float mx, mn;
   lane_minmax(make_row<PaddedRow>(rows, threadIdx.x), mx, mn);
-  encode_group<PaddedRow>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
+  encode_group<PaddedRow, 8>(sm, rows, lg, b, jg, g, y, sout, mx, mn, tail);
 }
 
 template <bool kDivide>
