@@ -37,9 +37,9 @@ METRIC = "compress / decompress / fused reduce-step GB/s (fp32 input) and % of B
 # expressed per value: DRAM traffic grows in proportion to the values processed, so a full-size launch is
 # this figure times its value count.  (Writes that are still in L2 when the kernel ends are not in it.)
 NCU_DRAM_BYTES_PER_VALUE = {
-    "ccoll_compress_kernel": (134.30e6 + 8.07e6) / 33554432,
+    "ccoll_compress_kernel": (134.30e6 + 7.25e6) / 33554432,
     "ccoll_decode_kernel": (58.74e6 + 79.48e6) / 33554432,
-    "ccoll_reduce_kernel": (194.11e6 + 157.51e6) / 33554432,
+    "ccoll_reduce_kernel": (193.68e6 + 158.67e6) / 33554432,
 }
 
 
