@@ -377,6 +377,9 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   const size_t Gc = groups_of(C);
   uint8_t* buf = ws->ptr + kOffStreams;
   uint64_t* bytes = reinterpret_cast<uint64_t*>(ws->ptr + kOffJobBytes);
+  // the root keeps its own data uncompressed (first, so that nothing stands between the two kernels below)
+  size_t own = (mode == CCOLL_BCAST) ? n : (C < n ? C : n);
+  if (own && cudaMemcpyAsync(out, root_in, 4 * own, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CCOLL_ERR_CUDA;
   // the root compresses every chunk exactly once
   uint32_t epoch;
   if ((rc = next_epoch(ws, s, &epoch)) != CCOLL_OK) return rc;
@@ -393,13 +396,13 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   b.state_stride = state_words((uint32_t)Gc);
   if (!launch_compress(b, (uint32_t)(Gc ? Gc : 1), (uint32_t)P, s)) return CCOLL_ERR_CUDA;
   if ((rc = check_launch()) != CCOLL_OK) return rc;
-  if (chunk_bytes &&
-      cudaMemcpyAsync(chunk_bytes, bytes, (size_t)P * sizeof(uint64_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-    return CCOLL_ERR_CUDA;
-  // the root keeps its own data uncompressed
-  size_t own = (mode == CCOLL_BCAST) ? n : (C < n ? C : n);
-  if (own && cudaMemcpyAsync(out, root_in, 4 * own, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CCOLL_ERR_CUDA;
-  if (P == 1 || Gc == 0) return CCOLL_OK;
+  auto report_sizes = [&]() -> int {
+    if (chunk_bytes &&
+        cudaMemcpyAsync(chunk_bytes, bytes, (size_t)P * sizeof(uint64_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+      return CCOLL_ERR_CUDA;
+    return CCOLL_OK;
+  };
+  if (P == 1 || Gc == 0) return report_sizes();
   DecodeBatch d;
   std::memset(&d, 0, sizeof(d));
   d.sin = buf;
@@ -411,15 +414,17 @@ int ccoll_bcast_sim(const float* root_in, float* out, size_t out_rank_stride, in
   d.n = n;
   d.P = P;
   d.status = reinterpret_cast<uint32_t*>(ws->ptr + kOffStatus);
+  // the receivers' grid directly behind the root's: it may fill the slots the compress grid's last wave leaves
   if (mode == CCOLL_BCAST) {
     d.skip_mode = 2;  // rank 0 is the root
-    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s)) return CCOLL_ERR_CUDA;
+    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, (uint32_t)P, s, /*behind_producer=*/true)) return CCOLL_ERR_CUDA;
   } else {
     d.skip_mode = 3;  // chunk 0 stays at the root
     d.scatter = 1;
-    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s)) return CCOLL_ERR_CUDA;
+    if (!launch_decode(d, (uint32_t)Gc, (uint32_t)P, 1, s, /*behind_producer=*/true)) return CCOLL_ERR_CUDA;
   }
-  return check_launch();
+  if ((rc = check_launch()) != CCOLL_OK) return rc;
+  return report_sizes();
 }
 
 int ccoll_bcast_sim_p2p(const float* root_in, float* out, size_t out_rank_stride, int P, size_t n, float abs_err_bound,
